@@ -1,0 +1,141 @@
+/*
+ * q8.h -- C ABI of the sm_100a int8 inference path of Q8BERT (arXiv 1910.06188).
+ *
+ * The library implements the inference mode of the paper's quantised layers (Sec. 3):
+ * symmetric linear quantisation to Int8 (Eq. 1, Eq. 2), per-tensor weight scale (Eq. 3),
+ * activation scale from an EMA of max|x| (Eq. 4) or computed per incoming tensor (Sec. 4.1),
+ * the Int8 x Int8 -> Int32 GEMM accumulated onto an Int32 bias, and the Int8 embedding lookup.
+ *
+ * Conventions that hold for every entry point
+ *   - All data pointers are DEVICE pointers on the current CUDA device unless a parameter says
+ *     "host".  The caller owns every buffer; the library never allocates or frees device memory.
+ *   - Tensors are dense row-major.  Activations X are [M, K], weights W / W_q are [N, K]
+ *     (out-features first, so Y = X W^T + b), outputs Y are [M, N].
+ *   - Scales are single fp32 values living in device memory, so no call forces a host sync.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue
+ *     work; they return after argument checks and launches.
+ *   - Argument errors are returned at once as a q8_status and nothing is launched.  Conditions
+ *     only the device can see (zero or non-finite max|x|, an out-of-range token id, a bounded
+ *     device-side wait that ran out) are OR-ed as bit (1 << code) into a device status word and
+ *     read back with q8_poll_status().  No kernel traps or spins without limit.
+ *   - float pointers must be 4-byte aligned; 16-byte alignment of X, Y, W_q (and K % 16 == 0)
+ *     selects the vectorised / tensor-core kernels, anything else runs the generic kernels
+ *     with identical results.
+ *   - Results are deterministic: the same inputs give bit-identical outputs.
+ */
+#ifndef Q8_H_
+#define Q8_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    Q8_OK = 0,
+    Q8_ERR_NULL = 1,      /* a required pointer is NULL */
+    Q8_ERR_SHAPE = 2,     /* negative size, K == 0, size beyond the supported range */
+    Q8_ERR_ALIGN = 3,     /* pointer not aligned to its element type / workspace not 256-byte aligned */
+    Q8_ERR_SCALE = 4,     /* device: max|x| was 0 or non-finite; scale forced to 1 */
+    Q8_ERR_INDEX = 5,     /* device: embedding id outside [0, V); that row is written as zeros */
+    Q8_ERR_OVERFLOW = 6,  /* K > 133144: K * 127^2 would not fit the Int32 accumulator */
+    Q8_ERR_WORKSPACE = 7, /* workspace smaller than q8_linear_workspace_bytes() */
+    Q8_ERR_TIMEOUT = 8,   /* device: a bounded wait inside the GEMM kernel expired */
+    Q8_ERR_CUDA = 9,      /* a CUDA runtime / driver call failed */
+    Q8_ERR_ARG = 10       /* invalid enum or parameter value (act, decay) */
+} q8_status;
+
+/* Largest reduction length for which the Int32 accumulator is exact: floor((2^31-1)/127^2). */
+#define Q8_MAX_K 133144
+
+/* Activation applied after dequantisation (Sec. 3 keeps GELU in FP32). */
+#define Q8_ACT_NONE 0
+#define Q8_ACT_GELU 1 /* y * Phi(y), erf form */
+
+/* Eq. 3 followed by Eq. 1 (one-time weight preparation; also used for embedding tables).
+ *   W      [N, K] fp32, read.
+ *   Wq     [N, K] int8, written: Clamp(nint(W * S_w), -127, 127).
+ *   S_w    1 fp32, written: 127 / max|W|  (1.0 and Q8_ERR_SCALE flagged if max|W| is 0 / non-finite).
+ *   dev_status  optional device status word (may be NULL), OR-ed into, never cleared.
+ * N == 0 or K == 0 is a no-op that writes S_w = 1. */
+q8_status q8_quantize_weight(const float *W, int64_t N, int64_t K, int8_t *Wq, float *S_w,
+                             int32_t *dev_status, void *stream);
+
+/* Eq. 1 on an activation tensor (flat, `numel` elements).
+ *   S_x != NULL: static scale (an Eq. 4 result), read.           S_x_used may be NULL.
+ *   S_x == NULL: dynamic scale of Sec. 4.1, S = 127 / max|X| over this tensor, written to
+ *                S_x_used (required; it also serves as the reduction scratch word).
+ *   Xq     int8 [numel], written. */
+q8_status q8_quantize_activation(const float *X, int64_t numel, const float *S_x, int8_t *Xq,
+                                 float *S_x_used, int32_t *dev_status, void *stream);
+
+/* Eq. 4: one calibration batch.  `state` is a q8_calibrate_state_bytes()-byte, 16-byte aligned,
+ * zero-initialised device block laid out as
+ *   { float ema; float S_x; int32 n_batches; uint32 scratch; int32 status; int32 pad[3]; }
+ * The first batch sets ema = max|X|; later ones do ema += (1 - decay) * (max|X| - ema) in fp32;
+ * then S_x = 127 / ema.  decay must lie in [0, 1); decay 0 reproduces the dynamic scale.
+ * &state->S_x can be passed as S_x to q8_linear. */
+q8_status q8_calibrate(const float *X, int64_t numel, float decay, void *state, void *stream);
+size_t q8_calibrate_state_bytes(void);
+
+/* The quantised fully-connected layer in inference mode (Sec. 3):
+ *   X_q = Quantize(X | S_x)  (Eq. 1);  acc = X_q W_q^T in Int32, accumulated onto the Int32 bias
+ *   b_q = Clamp(nint(b * fl32(S_x * S_w)), -(2^31-1), 2^31-1);  Y = (acc + b_q) / (S_x * S_w);
+ *   optional GELU.
+ *   X [M,K] fp32; Wq [N,K] int8 with its scale S_w (from q8_quantize_weight); bias [N] fp32 or NULL.
+ *   S_x: static activation scale, or NULL for the dynamic scale 127 / max|X| of Sec. 4.1.
+ *   act: Q8_ACT_NONE or Q8_ACT_GELU.      Y [M,N] fp32, written.
+ *   workspace: >= q8_linear_workspace_bytes(M,N,K) bytes, 256-byte aligned, caller-owned scratch
+ *     (status word at offset 0, then the quantised activation).  Its contents need not be
+ *     initialised; the status word is cleared at the start of every call.  Two calls that share
+ *     a workspace must be ordered on the stream.
+ *   dbg_Xq [M,K] int8 / dbg_acc [M,N] int32: optional (NULL to skip) copies of the quantised
+ *     activation and of acc + b_q, for bit-exact checks.
+ * M == 0 or N == 0 is a no-op.  K == 0 is Q8_ERR_SHAPE; K > Q8_MAX_K is Q8_ERR_OVERFLOW. */
+q8_status q8_linear(const float *X, const int8_t *Wq, const float *S_w, const float *S_x,
+                    const float *bias, int act, float *Y, int64_t M, int64_t N, int64_t K,
+                    void *workspace, size_t workspace_bytes, int8_t *dbg_Xq, int32_t *dbg_acc,
+                    void *stream);
+size_t q8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+/* Same layer on an activation that is already Int8 (the GEMM, bias, dequantise and activation
+ * steps only).  Xq [M,K] int8 and S_x (required) describe the quantised input.  dev_status is an
+ * optional status word that receives Q8_ERR_TIMEOUT. */
+q8_status q8_linear_q(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w,
+                      const float *bias, int act, float *Y, int64_t M, int64_t N, int64_t K,
+                      int32_t *dbg_acc, int32_t *dev_status, void *stream);
+
+/* q8_linear / q8_linear_q forced onto the generic (any shape, any alignment, CUDA-core) GEMM
+ * kernel that q8_linear uses by itself when K % 16 != 0 or an operand is not 16-byte aligned.
+ * Same arguments, same results; kept public as an on-device cross-check of the tensor-core kernel. */
+q8_status q8_linear_generic(const float *X, const int8_t *Wq, const float *S_w, const float *S_x,
+                            const float *bias, int act, float *Y, int64_t M, int64_t N, int64_t K,
+                            void *workspace, size_t workspace_bytes, int8_t *dbg_Xq,
+                            int32_t *dbg_acc, void *stream);
+
+/* Quantised embedding layer in inference mode (Sec. 3): gathers Int8 rows of the table and hands
+ * them to the FP32 consumer dequantised: out[t, :] = Eq[ids[t], :] / S_e.
+ *   ids [T] int32; Eq [V,H] int8; S_e 1 fp32; out [T,H] fp32 (written); rows_q [T,H] int8 optional
+ *   raw-row output (NULL to skip).  An id outside [0,V) yields a zero row and flags Q8_ERR_INDEX
+ *   in dev_status (optional). */
+q8_status q8_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,
+                       int64_t H, float *out, int8_t *rows_q, int32_t *dev_status, void *stream);
+
+/* Synchronises `stream`, reads the device status word at `dev_status` (a q8_linear workspace
+ * pointer works: the word sits at offset 0), clears it, and returns the lowest-numbered code
+ * whose bit was set (Q8_OK if none).  `raw_bits` (host pointer, may be NULL) receives the word. */
+q8_status q8_poll_status(void *dev_status, uint32_t *raw_bits, void *stream);
+
+const char *q8_status_string(q8_status s);
+
+/* Number of tile-CTAs and kernel launches the most recent q8_linear / q8_linear_q call on this
+ * host thread enqueued, and which GEMM kernel it chose (0 none, 1 tcgen05, 2 generic).
+ * Host-side bookkeeping for benchmarks; any pointer may be NULL. */
+void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *grid);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* Q8_H_ */

@@ -1,0 +1,233 @@
+"""ctypes binding of ``libq8.so``: same names as ``include/q8.h``, argument marshalling only.
+
+Every function takes torch tensors that already live on the CUDA device (torch supplies device
+memory and streams, nothing else), checks dtype / device / contiguity, passes raw pointers to
+the C ABI and raises :class:`Q8Error` on a non-zero status.  There is no CPU fallback: if the
+shared library is missing the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libq8.so")
+
+Q8_OK, Q8_ERR_NULL, Q8_ERR_SHAPE, Q8_ERR_ALIGN, Q8_ERR_SCALE, Q8_ERR_INDEX = 0, 1, 2, 3, 4, 5
+Q8_ERR_OVERFLOW, Q8_ERR_WORKSPACE, Q8_ERR_TIMEOUT, Q8_ERR_CUDA, Q8_ERR_ARG = 6, 7, 8, 9, 10
+Q8_ACT_NONE, Q8_ACT_GELU = 0, 1
+Q8_MAX_K = 133144
+
+# name -> (restype, argtypes); mirrors include/q8.h one to one.
+_vp, _i64, _sz, _int, _f = C.c_void_p, C.c_int64, C.c_size_t, C.c_int, C.c_float
+SIGNATURES = {
+    "q8_quantize_weight": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "q8_quantize_activation": (_int, [_vp, _i64, _vp, _vp, _vp, _vp, _vp]),
+    "q8_calibrate": (_int, [_vp, _i64, _f, _vp, _vp]),
+    "q8_calibrate_state_bytes": (_sz, []),
+    "q8_linear": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
+    "q8_linear_workspace_bytes": (_sz, [_i64, _i64, _i64]),
+    "q8_linear_q": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "q8_linear_generic": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
+    "q8_embedding": (_int, [_vp, _i64, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "q8_poll_status": (_int, [_vp, C.POINTER(C.c_uint32), _vp]),
+    "q8_status_string": (C.c_char_p, [_int]),
+    "q8_last_launch_info": (None, [C.POINTER(_int)] * 4),
+}
+
+_lib: Optional[C.CDLL] = None
+
+
+class Q8Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: q8_status {status} ({status_string(status)})")
+
+
+def load() -> C.CDLL:
+    """Loads libq8.so (built by ``python -m paper_1910_06188_b200.build``); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} not found: build the CUDA library first "
+                "(python -m paper_1910_06188_b200.build); there is no CPU fallback")
+        lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load().q8_status_string(int(status)).decode()
+
+
+# ---------------------------------------------------------------- marshalling helpers
+def _ptr(t: Optional[torch.Tensor], dtype: torch.dtype, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise TypeError(f"{name} must be contiguous")
+    return t.data_ptr()
+
+
+def _any_ptr(t: Optional[torch.Tensor], name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream or None
+    return int(stream) or None
+
+
+def _check(status: int, where: str) -> None:
+    if status != Q8_OK:
+        raise Q8Error(status, where)
+
+
+# ---------------------------------------------------------------- the calls
+def q8_quantize_weight(W: torch.Tensor, Wq: Optional[torch.Tensor] = None, S_w: Optional[torch.Tensor] = None,
+                       dev_status: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Eq. 3 + Eq. 1 on a weight (or embedding table) [N, K]; returns (W_q int8, S_w fp32[1])."""
+    N, K = W.shape
+    if Wq is None:
+        Wq = torch.empty((N, K), dtype=torch.int8, device=W.device)
+    if S_w is None:
+        S_w = torch.empty(1, dtype=torch.float32, device=W.device)
+    st = load().q8_quantize_weight(_ptr(W, torch.float32, "W"), N, K, _ptr(Wq, torch.int8, "Wq"),
+                                   _ptr(S_w, torch.float32, "S_w"), _ptr(dev_status, torch.int32, "dev_status"),
+                                   _stream(stream))
+    _check(st, "q8_quantize_weight")
+    return Wq, S_w
+
+
+def q8_quantize_activation(X: torch.Tensor, S_x: Optional[torch.Tensor] = None, Xq: Optional[torch.Tensor] = None,
+                           S_x_used: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                           stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Eq. 1 on an activation; S_x None selects the dynamic scale.  Returns (X_q, scale used)."""
+    if Xq is None:
+        Xq = torch.empty(X.shape, dtype=torch.int8, device=X.device)
+    if S_x is None and S_x_used is None:
+        S_x_used = torch.empty(1, dtype=torch.float32, device=X.device)
+    st = load().q8_quantize_activation(_ptr(X, torch.float32, "X"), X.numel(), _ptr(S_x, torch.float32, "S_x"),
+                                       _ptr(Xq, torch.int8, "Xq"), _ptr(S_x_used, torch.float32, "S_x_used"),
+                                       _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
+    _check(st, "q8_quantize_activation")
+    return Xq, (S_x_used if S_x_used is not None else S_x)
+
+
+def q8_calibrate_state_bytes() -> int:
+    return int(load().q8_calibrate_state_bytes())
+
+
+def new_calibrate_state(device="cuda") -> torch.Tensor:
+    """Zero-initialised Eq. 4 state block, viewed as int32 words: [ema, S_x, n_batches, scratch, status, ...]."""
+    return torch.zeros(q8_calibrate_state_bytes() // 4, dtype=torch.int32, device=device)
+
+
+def calibrate_S_x(state: torch.Tensor) -> torch.Tensor:
+    """fp32[1] view of the S_x word inside a calibrate state (usable as q8_linear's S_x)."""
+    return state.view(torch.float32)[1:2]
+
+
+def q8_calibrate(X: torch.Tensor, decay: float, state: torch.Tensor, stream=None) -> None:
+    st = load().q8_calibrate(_ptr(X, torch.float32, "X"), X.numel(), float(decay), _any_ptr(state, "state"),
+                             _stream(stream))
+    _check(st, "q8_calibrate")
+
+
+def q8_linear_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(load().q8_linear_workspace_bytes(M, N, K))
+
+
+def new_workspace(M: int, N: int, K: int, device="cuda") -> torch.Tensor:
+    return torch.empty(q8_linear_workspace_bytes(M, N, K), dtype=torch.uint8, device=device)
+
+
+def _linear(fn_name: str, X, Wq, S_w, S_x, bias, act, Y, workspace, dbg_Xq, dbg_acc, stream):
+    M, K = X.shape
+    N, K2 = Wq.shape
+    if K != K2:
+        raise ValueError(f"X is [M,{K}] but Wq is [N,{K2}]")
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float32, device=X.device)
+    if workspace is None:
+        workspace = new_workspace(M, N, K, X.device)
+    fn = getattr(load(), fn_name)
+    st = fn(_ptr(X, torch.float32, "X"), _ptr(Wq, torch.int8, "Wq"), _ptr(S_w, torch.float32, "S_w"),
+            _ptr(S_x, torch.float32, "S_x"), _ptr(bias, torch.float32, "bias"), int(act),
+            _ptr(Y, torch.float32, "Y"), M, N, K, _any_ptr(workspace, "workspace"),
+            workspace.numel() * workspace.element_size(), _ptr(dbg_Xq, torch.int8, "dbg_Xq"),
+            _ptr(dbg_acc, torch.int32, "dbg_acc"), _stream(stream))
+    _check(st, fn_name)
+    return Y
+
+
+def q8_linear(X, Wq, S_w, S_x=None, bias=None, act: int = Q8_ACT_NONE, Y=None, workspace=None, dbg_Xq=None,
+              dbg_acc=None, stream=None) -> torch.Tensor:
+    """Inference-mode quantised FC (Sec. 3): quantise X, Int8 GEMM, Int32 bias, dequantise, act."""
+    return _linear("q8_linear", X, Wq, S_w, S_x, bias, act, Y, workspace, dbg_Xq, dbg_acc, stream)
+
+
+def q8_linear_generic(X, Wq, S_w, S_x=None, bias=None, act: int = Q8_ACT_NONE, Y=None, workspace=None, dbg_Xq=None,
+                      dbg_acc=None, stream=None) -> torch.Tensor:
+    return _linear("q8_linear_generic", X, Wq, S_w, S_x, bias, act, Y, workspace, dbg_Xq, dbg_acc, stream)
+
+
+def q8_linear_q(Xq, S_x, Wq, S_w, bias=None, act: int = Q8_ACT_NONE, Y=None, dbg_acc=None, dev_status=None,
+                stream=None) -> torch.Tensor:
+    M, K = Xq.shape
+    N, K2 = Wq.shape
+    if K != K2:
+        raise ValueError(f"Xq is [M,{K}] but Wq is [N,{K2}]")
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float32, device=Xq.device)
+    st = load().q8_linear_q(_ptr(Xq, torch.int8, "Xq"), _ptr(S_x, torch.float32, "S_x"), _ptr(Wq, torch.int8, "Wq"),
+                            _ptr(S_w, torch.float32, "S_w"), _ptr(bias, torch.float32, "bias"), int(act),
+                            _ptr(Y, torch.float32, "Y"), M, N, K, _ptr(dbg_acc, torch.int32, "dbg_acc"),
+                            _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
+    _check(st, "q8_linear_q")
+    return Y
+
+
+def q8_embedding(ids, Eq, S_e, out=None, rows_q=None, dev_status=None, stream=None) -> torch.Tensor:
+    T = ids.numel()
+    V, H = Eq.shape
+    if out is None:
+        out = torch.empty((T, H), dtype=torch.float32, device=Eq.device)
+    st = load().q8_embedding(_ptr(ids, torch.int32, "ids"), T, _ptr(Eq, torch.int8, "Eq"),
+                             _ptr(S_e, torch.float32, "S_e"), V, H, _ptr(out, torch.float32, "out"),
+                             _ptr(rows_q, torch.int8, "rows_q"), _ptr(dev_status, torch.int32, "dev_status"),
+                             _stream(stream))
+    _check(st, "q8_embedding")
+    return out
+
+
+def q8_poll_status(dev_status: torch.Tensor, stream=None) -> Tuple[int, int]:
+    """Synchronises, reads and clears a device status word; returns (first status code, raw bits)."""
+    raw = C.c_uint32(0)
+    st = load().q8_poll_status(_any_ptr(dev_status, "dev_status"), C.byref(raw), _stream(stream))
+    return int(st), int(raw.value)
+
+
+def q8_last_launch_info() -> dict:
+    a, b, c, d = C.c_int(0), C.c_int(0), C.c_int(0), C.c_int(0)
+    load().q8_last_launch_info(C.byref(a), C.byref(b), C.byref(c), C.byref(d))
+    return dict(gemm_kernel=a.value, launches=b.value, block_n=c.value, grid=d.value)

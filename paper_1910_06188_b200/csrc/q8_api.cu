@@ -1,0 +1,280 @@
+// extern "C" entry points of libq8: argument validation, kernel selection and launches.
+// Nothing here computes; every step of the path runs in the kernels of the other files.
+
+#include <limits.h>
+
+#include "q8_internal.cuh"
+
+namespace q8 {
+
+LaunchInfo &last_launch_info()
+{
+    static thread_local LaunchInfo info;
+    return info;
+}
+
+namespace {
+
+inline bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+#define Q8_CUDA_TRY(expr)                      \
+    do {                                       \
+        cudaError_t e__ = (expr);              \
+        if (e__ != cudaSuccess) return Q8_ERR_CUDA; \
+    } while (0)
+
+// Eq. 1 with either a given scale or the dynamic one of Eq. 3 / Sec. 4.1 (scratch == output scale word).
+q8_status quantize_tensor(const float *X, int64_t numel, const float *S_given, int8_t *Xq, int8_t *Xq_copy,
+                          float *S_dyn, bool S_dyn_is_zero, int32_t *status, cudaStream_t s)
+{
+    LaunchInfo &li = last_launch_info();
+    const float *S = S_given;
+    if (S_given == nullptr) {
+        // The scale word first holds the float bits of the running maximum, then the scale itself.
+        if (!S_dyn_is_zero) Q8_CUDA_TRY(cudaMemsetAsync(S_dyn, 0, sizeof(float), s));
+        Q8_CUDA_TRY(launch_absmax(X, numel, reinterpret_cast<uint32_t *>(S_dyn), s));
+        Q8_CUDA_TRY(launch_scale_from_absmax(reinterpret_cast<const uint32_t *>(S_dyn), S_dyn, status, s));
+        li.launches += numel > 0 ? 2 : 1;
+        S = S_dyn;
+    }
+    Q8_CUDA_TRY(launch_quantize(X, numel, S, Xq, Xq_copy, s));
+    li.launches += numel > 0 ? 1 : 0;
+    return Q8_OK;
+}
+
+q8_status check_gemm_shape(int64_t M, int64_t N, int64_t K)
+{
+    if (M < 0 || N < 0 || K < 0) return Q8_ERR_SHAPE;
+    if (M == 0 || N == 0) return Q8_OK;
+    if (K == 0) return Q8_ERR_SHAPE;
+    if (K > Q8_MAX_K) return Q8_ERR_OVERFLOW;
+    if (M > (int64_t)INT_MAX || N > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
+    return Q8_OK;
+}
+
+q8_status run_gemm(const GemmArgs &g, bool force_generic, cudaStream_t s)
+{
+    if (!force_generic && tcgen05_gemm_supported(g)) {
+        Q8_CUDA_TRY(launch_gemm_tcgen05(g, s));
+    } else {
+        Q8_CUDA_TRY(launch_gemm_generic(g, s));
+    }
+    return Q8_OK;
+}
+
+q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
+                      float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
+                      int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic)
+{
+    last_launch_info() = LaunchInfo();
+    if (!X || !Wq || !S_w || !Y || !workspace) return Q8_ERR_NULL;
+    q8_status st = check_gemm_shape(M, N, K);
+    if (st != Q8_OK) return st;
+    if (act != Q8_ACT_NONE && act != Q8_ACT_GELU) return Q8_ERR_ARG;
+    if (!aligned_to(X, 4) || !aligned_to(Y, 4) || !aligned_to(S_w, 4) || (S_x && !aligned_to(S_x, 4)) ||
+        (bias && !aligned_to(bias, 4)) || (dbg_acc && !aligned_to(dbg_acc, 4)) || !aligned_to(workspace, 256))
+        return Q8_ERR_ALIGN;
+    if (workspace_bytes < q8_linear_workspace_bytes(M, N, K)) return Q8_ERR_WORKSPACE;
+    if (M == 0 || N == 0) return Q8_OK;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    WorkspaceHeader *hdr = static_cast<WorkspaceHeader *>(workspace);
+    int8_t *Xq = static_cast<int8_t *>(workspace) + kWorkspaceHeaderBytes;
+    Q8_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), s));
+
+    // Eq. 1, with the Sec. 4.1 dynamic scale when S_x is NULL (the header was just zeroed).
+    st = quantize_tensor(X, M * K, S_x, Xq, dbg_Xq, &hdr->S_x_dyn, true, &hdr->status, s);
+    if (st != Q8_OK) return st;
+
+    GemmArgs g;
+    g.Xq = Xq;
+    g.Wq = Wq;
+    g.S_x = S_x ? S_x : &hdr->S_x_dyn;
+    g.S_w = S_w;
+    g.bias = bias;
+    g.Y = Y;
+    g.dbg_acc = dbg_acc;
+    g.status = &hdr->status;
+    g.M = M;
+    g.N = N;
+    g.K = K;
+    g.act = act;
+    return run_gemm(g, force_generic, s);
+}
+
+}  // namespace
+}  // namespace q8
+
+using namespace q8;
+
+extern "C" {
+
+q8_status q8_quantize_weight(const float *W, int64_t N, int64_t K, int8_t *Wq, float *S_w, int32_t *dev_status,
+                             void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (!S_w) return Q8_ERR_NULL;
+    if (N < 0 || K < 0) return Q8_ERR_SHAPE;
+    if (N > 0 && K > 0 && (!W || !Wq)) return Q8_ERR_NULL;
+    if (N > 0 && K > 0 && N > (int64_t)LLONG_MAX / K) return Q8_ERR_SHAPE;
+    if (!aligned_to(W, 4) || !aligned_to(S_w, 4) || (dev_status && !aligned_to(dev_status, 4))) return Q8_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (N == 0 || K == 0) {
+        const float one = 1.0f;
+        Q8_CUDA_TRY(cudaMemcpyAsync(S_w, &one, sizeof(float), cudaMemcpyHostToDevice, s));
+        Q8_CUDA_TRY(cudaStreamSynchronize(s));  // `one` lives on this stack frame
+        return Q8_OK;
+    }
+    return quantize_tensor(W, N * K, nullptr, Wq, nullptr, S_w, false, dev_status, s);
+}
+
+q8_status q8_quantize_activation(const float *X, int64_t numel, const float *S_x, int8_t *Xq, float *S_x_used,
+                                 int32_t *dev_status, void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (numel < 0) return Q8_ERR_SHAPE;
+    if (numel > 0 && (!X || !Xq)) return Q8_ERR_NULL;
+    if (!S_x && !S_x_used) return Q8_ERR_NULL;
+    if (!aligned_to(X, 4) || (S_x && !aligned_to(S_x, 4)) || (S_x_used && !aligned_to(S_x_used, 4)) ||
+        (dev_status && !aligned_to(dev_status, 4)))
+        return Q8_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    q8_status st = quantize_tensor(X, numel, S_x, Xq, nullptr, S_x_used, false, dev_status, s);
+    if (st != Q8_OK) return st;
+    if (S_x && S_x_used && S_x_used != S_x)
+        Q8_CUDA_TRY(cudaMemcpyAsync(S_x_used, S_x, sizeof(float), cudaMemcpyDeviceToDevice, s));
+    return Q8_OK;
+}
+
+size_t q8_calibrate_state_bytes(void) { return sizeof(CalibState); }
+
+q8_status q8_calibrate(const float *X, int64_t numel, float decay, void *state, void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (!state) return Q8_ERR_NULL;
+    if (numel < 0) return Q8_ERR_SHAPE;
+    if (numel > 0 && !X) return Q8_ERR_NULL;
+    if (!(decay >= 0.0f && decay < 1.0f)) return Q8_ERR_ARG;
+    if (!aligned_to(X, 4) || !aligned_to(state, 16)) return Q8_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CalibState *st = static_cast<CalibState *>(state);
+    Q8_CUDA_TRY(launch_absmax(X, numel, &st->scratch_bits, s));
+    Q8_CUDA_TRY(launch_ema_update(st, decay, s));
+    last_launch_info().launches = numel > 0 ? 2 : 1;
+    return Q8_OK;
+}
+
+size_t q8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K)
+{
+    (void)N;
+    if (M < 0 || K < 0) return 0;
+    return kWorkspaceHeaderBytes + round_up((size_t)M * (size_t)K, 256);
+}
+
+q8_status q8_linear(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
+                    float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
+                    int8_t *dbg_Xq, int32_t *dbg_acc, void *stream)
+{
+    return linear_impl(X, Wq, S_w, S_x, bias, act, Y, M, N, K, workspace, workspace_bytes, dbg_Xq, dbg_acc, stream,
+                       false);
+}
+
+q8_status q8_linear_generic(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias,
+                            int act, float *Y, int64_t M, int64_t N, int64_t K, void *workspace,
+                            size_t workspace_bytes, int8_t *dbg_Xq, int32_t *dbg_acc, void *stream)
+{
+    return linear_impl(X, Wq, S_w, S_x, bias, act, Y, M, N, K, workspace, workspace_bytes, dbg_Xq, dbg_acc, stream,
+                       true);
+}
+
+q8_status q8_linear_q(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w, const float *bias,
+                      int act, float *Y, int64_t M, int64_t N, int64_t K, int32_t *dbg_acc, int32_t *dev_status,
+                      void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (!Xq || !S_x || !Wq || !S_w || !Y) return Q8_ERR_NULL;
+    q8_status st = check_gemm_shape(M, N, K);
+    if (st != Q8_OK) return st;
+    if (act != Q8_ACT_NONE && act != Q8_ACT_GELU) return Q8_ERR_ARG;
+    if (!aligned_to(Y, 4) || !aligned_to(S_w, 4) || !aligned_to(S_x, 4) || (bias && !aligned_to(bias, 4)) ||
+        (dbg_acc && !aligned_to(dbg_acc, 4)) || (dev_status && !aligned_to(dev_status, 4)))
+        return Q8_ERR_ALIGN;
+    if (M == 0 || N == 0) return Q8_OK;
+    GemmArgs g;
+    g.Xq = Xq;
+    g.Wq = Wq;
+    g.S_x = S_x;
+    g.S_w = S_w;
+    g.bias = bias;
+    g.Y = Y;
+    g.dbg_acc = dbg_acc;
+    g.status = dev_status;
+    g.M = M;
+    g.N = N;
+    g.K = K;
+    g.act = act;
+    return run_gemm(g, false, static_cast<cudaStream_t>(stream));
+}
+
+q8_status q8_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V, int64_t H,
+                       float *out, int8_t *rows_q, int32_t *dev_status, void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (T < 0 || V < 0 || H < 0) return Q8_ERR_SHAPE;
+    if (T == 0 || H == 0) return Q8_OK;
+    if (!ids || !S_e || !out) return Q8_ERR_NULL;
+    if (V > 0 && !Eq) return Q8_ERR_NULL;
+    if (V > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
+    if (T > (int64_t)LLONG_MAX / H) return Q8_ERR_SHAPE;
+    if (!aligned_to(ids, 4) || !aligned_to(S_e, 4) || !aligned_to(out, 4) ||
+        (dev_status && !aligned_to(dev_status, 4)))
+        return Q8_ERR_ALIGN;
+    Q8_CUDA_TRY(launch_embedding(ids, T, Eq, S_e, V, H, out, rows_q, dev_status, static_cast<cudaStream_t>(stream)));
+    last_launch_info().launches = 1;
+    return Q8_OK;
+}
+
+q8_status q8_poll_status(void *dev_status, uint32_t *raw_bits, void *stream)
+{
+    if (!dev_status) return Q8_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t bits = 0;
+    Q8_CUDA_TRY(cudaMemcpyAsync(&bits, dev_status, sizeof(bits), cudaMemcpyDeviceToHost, s));
+    Q8_CUDA_TRY(cudaMemsetAsync(dev_status, 0, sizeof(bits), s));
+    Q8_CUDA_TRY(cudaStreamSynchronize(s));
+    if (raw_bits) *raw_bits = bits;
+    for (int code = 1; code < 32; ++code)
+        if (bits & (1u << code)) return static_cast<q8_status>(code);
+    return Q8_OK;
+}
+
+const char *q8_status_string(q8_status s)
+{
+    switch (s) {
+        case Q8_OK: return "ok";
+        case Q8_ERR_NULL: return "required pointer is NULL";
+        case Q8_ERR_SHAPE: return "invalid or unsupported shape";
+        case Q8_ERR_ALIGN: return "pointer misaligned";
+        case Q8_ERR_SCALE: return "max|x| was zero or non-finite; scale forced to 1";
+        case Q8_ERR_INDEX: return "embedding id out of range";
+        case Q8_ERR_OVERFLOW: return "K too large for an exact Int32 accumulator";
+        case Q8_ERR_WORKSPACE: return "workspace too small";
+        case Q8_ERR_TIMEOUT: return "bounded device wait expired";
+        case Q8_ERR_CUDA: return "CUDA call failed";
+        case Q8_ERR_ARG: return "invalid argument value";
+    }
+    return "unknown status";
+}
+
+void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *grid)
+{
+    const LaunchInfo &li = last_launch_info();
+    if (gemm_kernel) *gemm_kernel = li.gemm_kernel;
+    if (launches) *launches = li.launches;
+    if (block_n) *block_n = li.block_n;
+    if (grid) *grid = li.grid;
+}
+
+}  // extern "C"

@@ -1,0 +1,293 @@
+// HBM-bound kernels of the Q8BERT inference path: max|x| reduction (Eq. 3 / Eq. 4 / Sec. 4.1),
+// the quantiser of Eq. 1, the EMA update of Eq. 4 and the Int8 embedding gather of Sec. 3.
+//
+// All of them stream their input once with 16-byte loads and stores; the grid is a multiple of
+// the SM count with a grid-stride loop so every SM keeps several independent loads in flight.
+
+#include "q8_internal.cuh"
+
+namespace q8 {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+int sm_count()
+{
+    static int n = [] {
+        int dev = 0, v = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        return v > 0 ? v : 148;
+    }();
+    return n;
+}
+
+int grid_for(int64_t work_items, int items_per_block, int blocks_per_sm)
+{
+    int64_t want = (work_items + items_per_block - 1) / items_per_block;
+    int64_t cap = (int64_t)sm_count() * blocks_per_sm;
+    if (want < 1) want = 1;
+    return (int)(want < cap ? want : cap);
+}
+
+// ------------------------------------------------------------------ max|x|
+__device__ __forceinline__ float absmax4(float m, float4 v)
+{
+    // fmaxf drops a NaN operand, so NaN entries are skipped; +-Inf propagates.
+    m = fmaxf(m, fabsf(v.x));
+    m = fmaxf(m, fabsf(v.y));
+    m = fmaxf(m, fabsf(v.z));
+    return fmaxf(m, fabsf(v.w));
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads) absmax_kernel(const float *__restrict__ x, int64_t n,
+                                                          uint32_t *__restrict__ bits)
+{
+    float m = 0.0f;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    if (VEC) {
+        const float4 *x4 = reinterpret_cast<const float4 *>(x);
+        const int64_t n4 = n >> 2;
+        int64_t i = tid;
+        // four independent 16-byte loads per iteration
+        for (; i + 3 * nthreads < n4; i += 4 * nthreads) {
+            float4 a = __ldg(x4 + i), b = __ldg(x4 + i + nthreads), c = __ldg(x4 + i + 2 * nthreads),
+                   d = __ldg(x4 + i + 3 * nthreads);
+            m = absmax4(absmax4(absmax4(absmax4(m, a), b), c), d);
+        }
+        for (; i < n4; i += nthreads) m = absmax4(m, __ldg(x4 + i));
+        for (int64_t j = (n4 << 2) + tid; j < n; j += nthreads) m = fmaxf(m, fabsf(x[j]));
+    } else {
+        for (int64_t j = tid; j < n; j += nthreads) m = fmaxf(m, fabsf(x[j]));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    __shared__ float warp_max[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0.0f;
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        // non-negative floats (and +Inf) order like their bit patterns
+        if (threadIdx.x == 0 && m > 0.0f) atomicMax(bits, __float_as_uint(m));
+    }
+}
+
+// S = 127 / max|.| (Eq. 3), in place over the scratch word when bits and S alias.
+__global__ void scale_from_absmax_kernel(const uint32_t *bits, float *S, int32_t *status)
+{
+    float a = __uint_as_float(*bits);
+    float s;
+    if (!(a > 0.0f) || isinf(a)) {
+        s = 1.0f;
+        if (status) atomicOr(status, 1 << Q8_ERR_SCALE);
+    } else {
+        s = __fdiv_rn(127.0f, a);
+    }
+    *S = s;
+}
+
+// ------------------------------------------------------------------ Eq. 1
+__device__ __forceinline__ int32_t quantize_one(float x, float S)
+{
+    // one rounded fp32 multiply, nearest-even integer (NaN -> 0, saturating), symmetric clamp
+    int32_t q = __float2int_rn(__fmul_rn(x, S));
+    return max(-127, min(127, q));
+}
+
+__device__ __forceinline__ uint32_t quantize_pack4(float4 v, float S)
+{
+    uint32_t a = (uint32_t)quantize_one(v.x, S) & 0xffu;
+    uint32_t b = (uint32_t)quantize_one(v.y, S) & 0xffu;
+    uint32_t c = (uint32_t)quantize_one(v.z, S) & 0xffu;
+    uint32_t d = (uint32_t)quantize_one(v.w, S) & 0xffu;
+    return a | (b << 8) | (c << 16) | (d << 24);
+}
+
+// VEC: a thread turns one 16-byte load (4 floats) into one 4-byte store, four of them in flight
+// per iteration; consecutive lanes touch consecutive addresses on both sides.
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restrict__ x, int64_t n,
+                                                            const float *__restrict__ S_ptr,
+                                                            int8_t *__restrict__ xq, int8_t *__restrict__ xq_copy)
+{
+    const float S = __ldg(S_ptr);
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    if (VEC) {
+        const float4 *x4 = reinterpret_cast<const float4 *>(x);
+        uint32_t *q4 = reinterpret_cast<uint32_t *>(xq);
+        uint32_t *c4 = reinterpret_cast<uint32_t *>(xq_copy);
+        const int64_t n4 = n >> 2;
+        int64_t i = tid;
+        for (; i + 3 * nthreads < n4; i += 4 * nthreads) {
+            float4 a = __ldg(x4 + i), b = __ldg(x4 + i + nthreads), c = __ldg(x4 + i + 2 * nthreads),
+                   d = __ldg(x4 + i + 3 * nthreads);
+            uint32_t qa = quantize_pack4(a, S), qb = quantize_pack4(b, S), qc = quantize_pack4(c, S),
+                     qd = quantize_pack4(d, S);
+            q4[i] = qa;
+            q4[i + nthreads] = qb;
+            q4[i + 2 * nthreads] = qc;
+            q4[i + 3 * nthreads] = qd;
+            if (xq_copy) {
+                c4[i] = qa;
+                c4[i + nthreads] = qb;
+                c4[i + 2 * nthreads] = qc;
+                c4[i + 3 * nthreads] = qd;
+            }
+        }
+        for (; i < n4; i += nthreads) {
+            uint32_t q = quantize_pack4(__ldg(x4 + i), S);
+            q4[i] = q;
+            if (xq_copy) c4[i] = q;
+        }
+        for (int64_t j = (n4 << 2) + tid; j < n; j += nthreads) {
+            int8_t q = (int8_t)quantize_one(x[j], S);
+            xq[j] = q;
+            if (xq_copy) xq_copy[j] = q;
+        }
+    } else {
+        for (int64_t j = tid; j < n; j += nthreads) {
+            int8_t q = (int8_t)quantize_one(x[j], S);
+            xq[j] = q;
+            if (xq_copy) xq_copy[j] = q;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ Eq. 4
+__global__ void ema_update_kernel(CalibState *st, float decay)
+{
+    float m = __uint_as_float(st->scratch_bits);
+    st->scratch_bits = 0u;
+    float ema;
+    if (st->n_batches == 0) {
+        ema = m;
+    } else {
+        // ema += (1 - d) * (m - ema), each operation rounded separately (no fused multiply-add)
+        float one_minus_d = __fsub_rn(1.0f, decay);
+        float step = __fmul_rn(one_minus_d, __fsub_rn(m, st->ema));
+        ema = __fadd_rn(st->ema, step);
+    }
+    st->ema = ema;
+    st->n_batches += 1;
+    if (!(ema > 0.0f) || isinf(ema)) {
+        st->S_x = 1.0f;
+        st->status |= 1 << Q8_ERR_SCALE;
+    } else {
+        st->S_x = __fdiv_rn(127.0f, ema);
+    }
+}
+
+// ------------------------------------------------------------------ Int8 embedding (Sec. 3)
+__device__ __forceinline__ float4 dequant4(uint32_t w, float inv)
+{
+    float4 f;
+    f.x = __fmul_rn((float)(int8_t)(w & 0xffu), inv);
+    f.y = __fmul_rn((float)(int8_t)((w >> 8) & 0xffu), inv);
+    f.z = __fmul_rn((float)(int8_t)((w >> 16) & 0xffu), inv);
+    f.w = __fmul_rn((float)(int8_t)(w >> 24), inv);
+    return f;
+}
+
+// VEC: one thread moves 4 table bytes (one 4-byte load) to one 16-byte store; consecutive lanes
+// cover consecutive pieces of a row, so a warp reads 128 and writes 512 contiguous bytes.
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads) embedding_kernel(const int32_t *__restrict__ ids, int64_t T,
+                                                             const int8_t *__restrict__ Eq,
+                                                             const float *__restrict__ S_e, int64_t V, int64_t H,
+                                                             float *__restrict__ out, int8_t *__restrict__ rows_q,
+                                                             int32_t *__restrict__ status)
+{
+    const float inv = __fdiv_rn(1.0f, __ldg(S_e));
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    if (VEC) {
+        const int64_t per_row = H >> 2;
+        const int64_t total = T * per_row;
+        for (int64_t w = tid; w < total; w += nthreads) {
+            const int64_t t = w / per_row, c = w - t * per_row;
+            const int64_t id = __ldg(ids + t);
+            uint32_t q = 0u;
+            if (id >= 0 && id < V) {
+                q = __ldg(reinterpret_cast<const uint32_t *>(Eq + id * H) + c);
+            } else if (c == 0 && status) {
+                atomicOr(status, 1 << Q8_ERR_INDEX);
+            }
+            __stcs(reinterpret_cast<float4 *>(out) + w, dequant4(q, inv));
+            if (rows_q) reinterpret_cast<uint32_t *>(rows_q)[w] = q;
+        }
+    } else {
+        const int64_t total = T * H;
+        for (int64_t e = tid; e < total; e += nthreads) {
+            const int64_t t = e / H, h = e - t * H;
+            const int64_t id = __ldg(ids + t);
+            int8_t q = 0;
+            if (id >= 0 && id < V) {
+                q = Eq[id * H + h];
+            } else if (h == 0 && status) {
+                atomicOr(status, 1 << Q8_ERR_INDEX);
+            }
+            out[e] = __fmul_rn((float)q, inv);
+            if (rows_q) rows_q[e] = q;
+        }
+    }
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+cudaError_t launch_absmax(const float *x, int64_t n, uint32_t *bits, cudaStream_t s)
+{
+    if (n <= 0) return cudaSuccess;
+    if (aligned16(x)) {
+        absmax_kernel<true><<<grid_for(n >> 2, kThreads * 4, 8), kThreads, 0, s>>>(x, n, bits);
+    } else {
+        absmax_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, bits);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scale_from_absmax(const uint32_t *bits, float *S, int32_t *status, cudaStream_t s)
+{
+    scale_from_absmax_kernel<<<1, 1, 0, s>>>(bits, S, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy, cudaStream_t s)
+{
+    if (n <= 0) return cudaSuccess;
+    if (aligned16(x) && aligned16(xq) && (xq_copy == nullptr || aligned16(xq_copy))) {
+        quantize_kernel<true><<<grid_for((n + 3) >> 2, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy);
+    } else {
+        quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ema_update(CalibState *st, float decay, cudaStream_t s)
+{
+    ema_update_kernel<<<1, 1, 0, s>>>(st, decay);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,
+                             int64_t H, float *out, int8_t *rows_q, int32_t *status, cudaStream_t s)
+{
+    if (T <= 0 || H <= 0) return cudaSuccess;
+    const bool vec = (H % 4 == 0) && aligned16(Eq) && aligned16(out) && (rows_q == nullptr || aligned16(rows_q));
+    if (vec) {
+        embedding_kernel<true><<<grid_for(T * (H >> 2), kThreads * 2, 8), kThreads, 0, s>>>(ids, T, Eq, S_e, V, H, out,
+                                                                                      rows_q, status);
+    } else {
+        embedding_kernel<false><<<grid_for(T * H, kThreads, 8), kThreads, 0, s>>>(ids, T, Eq, S_e, V, H, out,
+                                                                                 rows_q, status);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace q8

@@ -1,0 +1,92 @@
+// Internal declarations shared by the translation units of libq8 (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "q8.h"
+
+namespace q8 {
+
+// Layout of the head of a q8_linear workspace.
+struct WorkspaceHeader {
+    int32_t status;  // OR of (1 << q8_status) bits raised by kernels
+    float S_x_dyn;   // dynamic mode: first the float bits of max|X| (atomicMax scratch), then 127 / max|X|
+    int32_t pad[2];
+};
+constexpr size_t kWorkspaceHeaderBytes = 256;
+
+// Device block behind q8_calibrate (Eq. 4 running state).
+struct CalibState {
+    float ema;
+    float S_x;
+    int32_t n_batches;
+    uint32_t scratch_bits;
+    int32_t status;
+    int32_t pad[3];
+};
+
+struct GemmArgs {
+    const int8_t *Xq;   // [M,K]
+    const int8_t *Wq;   // [N,K]
+    const float *S_x;   // device scalar
+    const float *S_w;   // device scalar
+    const float *bias;  // [N] or nullptr
+    float *Y;           // [M,N]
+    int32_t *dbg_acc;   // [M,N] or nullptr
+    int32_t *status;    // device status word or nullptr
+    int64_t M, N, K;
+    int act;
+};
+
+struct LaunchInfo {
+    int gemm_kernel = 0;  // 0 none, 1 tcgen05, 2 generic
+    int launches = 0;
+    int block_n = 0;
+    int grid = 0;
+};
+LaunchInfo &last_launch_info();
+
+// ---- elementwise / reduction launchers (q8_elementwise.cu) ----
+// max|x| folded into *bits (must hold 0 or an earlier maximum) with atomicMax on the float bits.
+cudaError_t launch_absmax(const float *x, int64_t n, uint32_t *bits, cudaStream_t s);
+// *S = 127 / float(*bits) in place (bits and S may alias); flags Q8_ERR_SCALE on 0 / non-finite.
+cudaError_t launch_scale_from_absmax(const uint32_t *bits, float *S, int32_t *status, cudaStream_t s);
+cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy,
+                            cudaStream_t s);
+cudaError_t launch_ema_update(CalibState *st, float decay, cudaStream_t s);
+cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,
+                             int64_t H, float *out, int8_t *rows_q, int32_t *status, cudaStream_t s);
+
+// ---- GEMM launchers ----
+bool tcgen05_gemm_supported(const GemmArgs &a);
+cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s);  // q8_gemm_sm100.cu
+cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_generic.cu
+
+// ---- epilogue arithmetic shared by both GEMM kernels ----
+// Bias quantised at the product scale: Clamp(nint(b * S_out), -(2^31-1), 2^31-1).
+__device__ __forceinline__ int32_t quantize_bias(float b, float S_out)
+{
+    // cvt.rni saturates at the int32 range and maps NaN to 0; only INT_MIN needs the symmetric clamp.
+    int32_t q = __float2int_rn(__fmul_rn(b, S_out));
+    return max(q, -2147483647);
+}
+
+__device__ __forceinline__ float gelu_erf(float y)
+{
+    return 0.5f * y * (1.0f + erff(y * 0.70710678118654752440f));
+}
+
+// acc + b_q in Int32 (two's-complement wrap), dequantised with the reciprocal of the product scale.
+__device__ __forceinline__ float finish_output(int32_t acc_plus_bias, float inv_S_out, int act)
+{
+    float y = __fmul_rn(__int2float_rn(acc_plus_bias), inv_S_out);
+    return act == Q8_ACT_GELU ? gelu_erf(y) : y;
+}
+
+__device__ __forceinline__ int32_t add_wrap(int32_t a, int32_t b)
+{
+    return (int32_t)((uint32_t)a + (uint32_t)b);
+}
+
+}  // namespace q8
