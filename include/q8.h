@@ -75,7 +75,7 @@ q8_status q8_quantize_activation(const float *X, int64_t numel, const float *S_x
  * zero-initialised device block laid out as
  *   { float ema; float S_x; int32 n_batches; uint32 scratch; int32 status; int32 pad[3]; }
  * The first batch sets ema = max|X|; later ones do ema += (1 - decay) * (max|X| - ema) in fp32;
- * then S_x = 127 / ema.  decay must lie in [0, 1); decay 0 reproduces the dynamic scale.
+ * then S_x = 127 / ema.  decay must lie in [0, 1); decay 0 tracks the last batch (the dynamic scale, up to one fp32 rounding).
  * &state->S_x can be passed as S_x to q8_linear. */
 q8_status q8_calibrate(const float *X, int64_t numel, float decay, void *state, void *stream);
 size_t q8_calibrate_state_bytes(void);

@@ -84,10 +84,15 @@ def test_calibrate_matches_oracle_ema():
 
 def test_calibrate_decay_zero_is_dynamic_and_zero_batch_flags():
     state = q8.new_calibrate_state()
+    ref = o.EmaState()
     for i, g in enumerate((3.0, 0.5, 7.0)):
         x = synth.activation(8, 40, seed=310 + i) * np.float32(g)
         q8.q8_calibrate(dev(x), 0.0, state)
-        assert state.view(torch.float32)[1].item() == np.float32(127.0) / o.absmax(x)
+        ref.update(o.absmax(x), 0.0)
+        got = state.view(torch.float32)[1].item()
+        assert np.float32(got) == ref.S_x                      # same fp32 steps as the oracle
+        # decay 0 tracks the last batch: ema + 1*(m - ema) is m up to one fp32 rounding
+        assert abs(got - 127.0 / float(o.absmax(x))) <= 4e-7 * got
     state = q8.new_calibrate_state()
     q8.q8_calibrate(torch.zeros(100, device="cuda"), 0.9, state)
     assert state[4].item() == 1 << q8.Q8_ERR_SCALE and state.view(torch.float32)[1].item() == 1.0
