@@ -1,0 +1,426 @@
+#!/usr/bin/env python
+"""Benchmark of the int8 inference path of Q8BERT on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic BERT-shaped input: the
+Int8 embedding gather for the batch's tokens, then for each of the four fully-connected layers of
+an encoder block (QKV, attention-out, FFN1 + GELU, FFN2) the activation quantiser (Eq. 1, static
+scale from Eq. 4) followed by the tcgen05 Int8 GEMM with its fused bias / dequantise / GELU
+epilogue.  Weight quantisation (Eq. 3) and scale calibration (Eq. 4) are one-time set-up and are
+not timed.
+
+    python bench.py --gpus 1 --steps K --warmup W            # this library
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, bounded sample
+
+Prints ONE JSON line (rank 0).  `value` is TOPS (2*M*N*K summed over the four GEMMs, divided by the
+step time) with inputs resident in HBM; `e2e` is the same metric with host buffers and the
+host<->device copies inside the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1910_06188_b200 import synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (config index, model dims, description)
+    "bert_large_fc": (4, synth.BERT_LARGE, "BERT-Large FC set, batch 64 x seq 384 (M=24576 tokens)"),
+    "bert_base_fc": (2, synth.BERT_BASE, "BERT-Base FC set, batch 32 x seq 128 (M=4096 tokens)"),
+}
+NOMINAL_INT8_OVER_BF16 = 2.0  # dense tensor peak ratio int8 : bf16 (4.5 : 2.25 POPS nominal)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def make_layers(cfg_index: int, dims: dict):
+    """Host tensors of the four FC layers: activation, calibration batch, weight, bias."""
+    M = dims["batch"] * dims["seq"]
+    layers = []
+    for i, (name, K, N, act) in enumerate(synth.fc_set(dims["hidden"], dims["ffn"])):
+        layers.append(dict(
+            name=name, M=M, K=K, N=N, act=act,
+            X=synth.activation(M, K, synth.seed_for(cfg_index, 10 * i)),
+            calib=synth.activation(M, K, synth.seed_for(cfg_index, 10 * i + 1)),
+            W=synth.weight(N, K, synth.seed_for(cfg_index, 10 * i + 2)),
+            b=synth.bias(N, synth.seed_for(cfg_index, 10 * i + 3)),
+        ))
+    return M, layers
+
+
+def total_ops(layers):
+    return sum(2.0 * L["M"] * L["N"] * L["K"] for L in layers)
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                bits = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, v in names.items():
+                    if bits & v:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+# --------------------------------------------------------------------------- the CPU oracle arm
+def run_reference(args):
+    """Times the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from oracle import q8_oracle as o  # the one place besides cpu_baseline where bench.py runs the oracle
+
+    cfg_index, dims, desc = WORKLOADS[args.workload]
+    rows = args.reference_rows
+    layers = []
+    for i, (name, K, N, act) in enumerate(synth.fc_set(dims["hidden"], dims["ffn"])):
+        X = synth.activation(rows, K, synth.seed_for(cfg_index, 10 * i))
+        W = synth.weight(N, K, synth.seed_for(cfg_index, 10 * i + 2))
+        b = synth.bias(N, synth.seed_for(cfg_index, 10 * i + 3))
+        Wq, S_w, _ = o.quantize_weight(W)
+        S_x, _ = o.scale_from_absmax(o.absmax(X))
+        layers.append(dict(M=rows, K=K, N=N, act=act, X=X, Wq=Wq, S_w=S_w, S_x=S_x, b=b))
+    ops = total_ops(layers)
+
+    def step():
+        for L in layers:
+            o.linear(L["X"], L["Wq"], L["S_w"], L["S_x"], L["b"], L["act"])
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = ops / dt / 1e12
+    cores = os.cpu_count()
+    sample = f"{rows} of {dims['batch'] * dims['seq']} token rows of each of the 4 FC layers per step"
+    line = {
+        "impl": "reference", "metric": "q8_linear_int8_tops", "value": value, "unit": "TOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": args.workload, "description": desc, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# --------------------------------------------------------------------------- this library
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_1910_06188_b200 import binding as q8
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    q8.load()
+
+    cfg_index, dims, desc = WORKLOADS[args.workload]
+    # weak scaling: every rank owns one full batch of M tokens (rows are independent given static
+    # scales, so there is no data-path collective); rank r draws its batch from its own seeds.
+    M, layers = make_layers(cfg_index + 100 * rank, dims)
+    if args.layers:
+        keep = set(args.layers.split(","))
+        layers = [L for L in layers if L["name"] in keep]
+    ops = total_ops(layers)
+    H, V = dims["hidden"], dims["vocab"]
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream()
+
+    # ---- one-time set-up (not timed): Eq. 3 weights, Eq. 4 scales, embedding table
+    for L in layers:
+        L["Xd"] = torch.from_numpy(L["X"]).to(dev)
+        L["bd"] = torch.from_numpy(L["b"]).to(dev)
+        L["Wq"], L["S_w"] = q8.q8_quantize_weight(torch.from_numpy(L["W"]).to(dev))
+        state = q8.new_calibrate_state(dev)
+        q8.q8_calibrate(torch.from_numpy(L["calib"]).to(dev), 0.9999, state)
+        L["S_x"] = q8.calibrate_S_x(state).clone()
+        L["Y"] = torch.empty((L["M"], L["N"]), dtype=torch.float32, device=dev)
+        L["ws"] = q8.new_workspace(L["M"], L["N"], L["K"], dev)
+        L["Xq"] = torch.empty((L["M"], L["K"]), dtype=torch.int8, device=dev)
+        del L["calib"], L["W"]
+    E = synth.embedding_table(V, H, synth.seed_for(cfg_index, 90))
+    Eq, S_e = q8.q8_quantize_weight(torch.from_numpy(E).to(dev))
+    ids = torch.from_numpy(synth.token_ids(M, V, synth.seed_for(cfg_index + 100 * rank, 91))).to(dev)
+    emb_out = torch.empty((M, H), dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+
+    launches_per_step = 0
+
+    def step():
+        nonlocal launches_per_step
+        n = 0
+        q8.q8_embedding(ids, Eq, S_e, out=emb_out)
+        n += q8.q8_last_launch_info()["launches"]
+        for L in layers:
+            q8.q8_linear(L["Xd"], L["Wq"], L["S_w"], L["S_x"], L["bd"], L["act"], Y=L["Y"], workspace=L["ws"])
+            n += q8.q8_last_launch_info()["launches"]
+        launches_per_step = n
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    for L in layers:
+        code, bits = q8.q8_poll_status(L["ws"])
+        if code != q8.Q8_OK:
+            raise SystemExit(f"device status {code} ({q8.status_string(code)}) on layer {L['name']}")
+
+    # ---- timed region: K whole steps, device time, max over ranks
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    with sampler:
+        barrier()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            step()
+        ev1.record(stream)
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+
+        # ---- per-kernel pass (same launches, events around each kernel): roofline of the dominant kernel
+        nl = len(layers)
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(nl)]
+        t_quant, t_gemm = [0.0] * nl, [0.0] * nl
+        ev_e0, ev_e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_emb = 0.0
+        ksteps = 0 if args.profile_mode else min(args.steps, 50)
+        for _ in range(ksteps):
+            ev_e0.record(stream)
+            q8.q8_embedding(ids, Eq, S_e, out=emb_out)
+            ev_e1.record(stream)
+            for i, L in enumerate(layers):
+                evs[i][0].record(stream)
+                q8.q8_quantize_activation(L["Xd"], L["S_x"], Xq=L["Xq"])
+                evs[i][1].record(stream)
+                q8.q8_linear_q(L["Xq"], L["S_x"], L["Wq"], L["S_w"], L["bd"], L["act"], Y=L["Y"])
+                evs[i][2].record(stream)
+            torch.cuda.synchronize()
+            t_emb += ev_e0.elapsed_time(ev_e1)
+            for i in range(nl):
+                t_quant[i] += evs[i][0].elapsed_time(evs[i][1])
+                t_gemm[i] += evs[i][1].elapsed_time(evs[i][2])
+    clocks = sampler.summary()
+    if args.profile_mode:
+        if rank == 0:
+            print(json.dumps({"profile_mode": True, "ms_per_step": ms / args.steps, "steps": args.steps}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * ops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: host buffers, H2D of every input and D2H of every output inside the timed region
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    host_in = [torch.from_numpy(L["X"]).pin_memory() for L in layers]
+    host_ids = ids.cpu().pin_memory()
+    host_out = [torch.empty((L["M"], L["N"]), dtype=torch.float32).pin_memory() for L in layers]
+    host_emb = torch.empty((M, H), dtype=torch.float32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host_in) + host_ids.numel() * 4
+    d2h = sum(t.numel() * t.element_size() for t in host_out) + host_emb.numel() * 4
+
+    def e2e_step():
+        ids.copy_(host_ids, non_blocking=True)
+        q8.q8_embedding(ids, Eq, S_e, out=emb_out)
+        host_emb.copy_(emb_out, non_blocking=True)
+        for L, hi, ho in zip(layers, host_in, host_out):
+            L["Xd"].copy_(hi, non_blocking=True)
+            q8.q8_linear(L["Xd"], L["Wq"], L["S_w"], L["S_x"], L["bd"], L["act"], Y=L["Y"], workspace=L["ws"])
+            ho.copy_(L["Y"], non_blocking=True)
+
+    e2e_step()
+    barrier()
+    ev0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record(stream)
+    barrier()
+    e2e_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * ops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant kernel (the tcgen05 GEMM, launched once per FC layer)
+    peaks, peak_kind = load_peaks()
+    int8_peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"])) * NOMINAL_INT8_OVER_BF16
+    hbm_peak = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+    gemm_ms = [t / ksteps for t in t_gemm]
+    quant_ms = [t / ksteps for t in t_quant]
+    gemm_ops = [2.0 * L["M"] * L["N"] * L["K"] for L in layers]
+    gemm_bytes = [L["M"] * L["K"] + L["N"] * L["K"] + 4 * L["N"] + 4 * L["M"] * L["N"] for L in layers]
+    achieved = sum(gemm_ops) / (sum(gemm_ms) * 1e-3) / 1e12
+    by_layer = []
+    for L, gm, qm, go, gb in zip(layers, gemm_ms, quant_ms, gemm_ops, gemm_bytes):
+        by_layer.append({
+            "layer": L["name"], "M": L["M"], "K": L["K"], "N": L["N"],
+            "gemm_us": gm * 1e3, "gemm_tops": go / (gm * 1e-3) / 1e12, "gemm_frac_int8_peak": go / (gm * 1e-3) / 1e12 / int8_peak,
+            "gemm_gbs": gb / (gm * 1e-3) / 1e9, "gemm_frac_hbm": gb / (gm * 1e-3) / 1e9 / hbm_peak,
+            "quantize_us": qm * 1e3, "quantize_gbs": 5.0 * L["M"] * L["K"] / (qm * 1e-3) / 1e9,
+            "quantize_frac_hbm": 5.0 * L["M"] * L["K"] / (qm * 1e-3) / 1e9 / hbm_peak,
+        })
+    emb_ms = t_emb / ksteps
+    emb_bytes = 5.0 * M * H + 4.0 * M
+    roofline = {
+        "kernel": "gemm_tcgen05_kernel (4 launches per step, one per FC layer)",
+        "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
+        "traffic": None,
+        "peak_source": f"2 x bf16_tflops_sustained of {peak_kind} (nominal int8:bf16 dense ratio)",
+        "frac_of_nominal_4500": achieved / 4500.0,
+        "by_layer": by_layer,
+        "embedding": {"us": emb_ms * 1e3, "gbs": emb_bytes / (emb_ms * 1e-3) / 1e9,
+                      "frac_hbm": emb_bytes / (emb_ms * 1e-3) / 1e9 / hbm_peak},
+    }
+
+    # ---- CPU oracle on a bounded sample of the same workload (rank 0, N=1 only)
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import q8_oracle as o
+        rows = args.cpu_rows
+        t0 = time.perf_counter()
+        for L in layers:
+            Wq_h = L["Wq"].cpu().numpy()
+            o.linear(L["X"][:rows], Wq_h, float(L["S_w"].item()), float(L["S_x"].item()), L["b"], L["act"])
+        dt = time.perf_counter() - t0
+        sample_ops = sum(2.0 * rows * L["N"] * L["K"] for L in layers)
+        cpu_baseline = {
+            "value": sample_ops / dt / 1e12, "unit": "TOPS", "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"first {rows} of {M} token rows of each of the 4 FC layers, once ({dt:.1f} s)",
+        }
+
+    line = {
+        "metric": "q8_linear_int8_tops", "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {
+            "workload": args.workload, "description": desc, "tokens_per_step": M * world,
+            "tokens_per_s": M * world / (ms_per_step * 1e-3),
+            "l2": "inputs larger than L2 (each step reads ~0.9 GB and writes ~1.0 GB; L2 is 126 MB)",
+            "step": "q8_embedding + 4 x q8_linear (quantise, tcgen05 GEMM, fused epilogue), static scales",
+        },
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline,
+        "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="bert_large_fc")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-rows", type=int, default=2048, help="token rows per layer for the cpu_baseline sample")
+    ap.add_argument("--reference-rows", type=int, default=256, help="token rows per layer per step for --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", default="", help="comma list of FC layers to keep (qkv,attn_out,ffn1,ffn2); default all")
+    ap.add_argument("--profile-mode", action="store_true",
+                    help="only warm-up + timed steps (no per-kernel pass, e2e or CPU baseline): for ncu captures")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
