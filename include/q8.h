@@ -130,10 +130,17 @@ q8_status q8_poll_status(void *dev_status, uint32_t *raw_bits, void *stream);
 
 const char *q8_status_string(q8_status s);
 
-/* Number of tile-CTAs and kernel launches the most recent q8_linear / q8_linear_q call on this
- * host thread enqueued, and which GEMM kernel it chose (0 none, 1 tcgen05, 2 generic).
- * Host-side bookkeeping for benchmarks; any pointer may be NULL. */
-void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *grid);
+/* What the most recent call on this host thread enqueued: which GEMM kernel it chose (0 none,
+ * 1 tcgen05, 2 generic), how many kernels it launched, the tile width, the grid size and how many
+ * CTAs share one tile (2 = cta_group::2 pairs).  Host-side bookkeeping for benchmarks and tests;
+ * any pointer may be NULL. */
+void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *grid, int *ctas);
+
+/* Tuning / test hook: force the tile shape of the tcgen05 GEMM for later calls in this process.
+ * (block_n, ctas) = (0, 0) restores the automatic choice; otherwise ctas = 1 with block_n in
+ * {32, 64, 128, 256} (one SM per 128 x block_n tile) or ctas = 2 with block_n = 256 (a pair of
+ * SMs per 256 x 256 tile).  Results do not depend on the choice.  Not thread-safe. */
+q8_status q8_tune_gemm_tile(int block_n, int ctas);
 
 #ifdef __cplusplus
 }

@@ -35,7 +35,8 @@ SIGNATURES = {
     "q8_embedding": (_int, [_vp, _i64, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _vp]),
     "q8_poll_status": (_int, [_vp, C.POINTER(C.c_uint32), _vp]),
     "q8_status_string": (C.c_char_p, [_int]),
-    "q8_last_launch_info": (None, [C.POINTER(_int)] * 4),
+    "q8_last_launch_info": (None, [C.POINTER(_int)] * 5),
+    "q8_tune_gemm_tile": (_int, [_int, _int]),
 }
 
 _lib: Optional[C.CDLL] = None
@@ -228,6 +229,11 @@ def q8_poll_status(dev_status: torch.Tensor, stream=None) -> Tuple[int, int]:
 
 
 def q8_last_launch_info() -> dict:
-    a, b, c, d = C.c_int(0), C.c_int(0), C.c_int(0), C.c_int(0)
-    load().q8_last_launch_info(C.byref(a), C.byref(b), C.byref(c), C.byref(d))
-    return dict(gemm_kernel=a.value, launches=b.value, block_n=c.value, grid=d.value)
+    a, b, c, d, e = C.c_int(0), C.c_int(0), C.c_int(0), C.c_int(0), C.c_int(0)
+    load().q8_last_launch_info(C.byref(a), C.byref(b), C.byref(c), C.byref(d), C.byref(e))
+    return dict(gemm_kernel=a.value, launches=b.value, block_n=c.value, grid=d.value, ctas=e.value)
+
+
+def q8_tune_gemm_tile(block_n: int = 0, ctas: int = 0) -> None:
+    """Forces the tcgen05 GEMM tile shape for later calls ((0, 0) = automatic)."""
+    _check(load().q8_tune_gemm_tile(int(block_n), int(ctas)), "q8_tune_gemm_tile")

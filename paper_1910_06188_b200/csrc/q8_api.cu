@@ -268,13 +268,24 @@ const char *q8_status_string(q8_status s)
     return "unknown status";
 }
 
-void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *grid)
+void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *grid, int *ctas)
 {
     const LaunchInfo &li = last_launch_info();
     if (gemm_kernel) *gemm_kernel = li.gemm_kernel;
     if (launches) *launches = li.launches;
     if (block_n) *block_n = li.block_n;
     if (grid) *grid = li.grid;
+    if (ctas) *ctas = li.ctas;
+}
+
+q8_status q8_tune_gemm_tile(int block_n, int ctas)
+{
+    const bool automatic = block_n == 0 && ctas == 0;
+    const bool single = ctas == 1 && (block_n == 32 || block_n == 64 || block_n == 128 || block_n == 256);
+    const bool pair = ctas == 2 && block_n == 256;
+    if (!automatic && !single && !pair) return Q8_ERR_ARG;
+    set_gemm_tile_override(block_n, ctas);
+    return Q8_OK;
 }
 
 }  // extern "C"

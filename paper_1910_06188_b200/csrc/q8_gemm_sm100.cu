@@ -5,14 +5,20 @@
 //
 //   warp 0      TMA producer: 128-byte-swizzled K-major tiles of X_q [M,K] and W_q [N,K] go
 //               global -> shared through a ring of mbarrier-guarded stages
-//   warp 1      MMA issuer: one lane issues tcgen05.mma kind::i8 (128 x BLOCK_N x 32 per
-//               instruction); Int32 accumulators live in TMEM, double buffered
-//   warps 2..   epilogue: tcgen05.ld the accumulator, add b_q, convert, scale, GELU, store fp32
+//   warp 1      MMA issuer: one lane issues tcgen05.mma kind::i8; Int32 accumulators live in
+//               TMEM, double buffered
+//   warps 2..9  epilogue: tcgen05.ld the accumulator, add b_q, convert, scale, GELU, stage the
+//               fp32 block in swizzled shared memory and write it with a TMA store
 //
-// The kernel is persistent (one CTA per SM walks a static tile list), so the epilogue of tile i
-// overlaps the main loop of tile i+1.  No cluster multicast is used anywhere.  Every wait on an
-// mbarrier is bounded: after ~2 s the CTA raises Q8_ERR_TIMEOUT in the status word, all roles
-// leave their loops, in-flight copies are drained and TMEM is released before the CTA exits.
+// Two shapes of the same kernel: CTAS = 1 (one SM per 128 x BLOCK_N tile) for small problems, and
+// CTAS = 2 (cta_group::2: a pair of SMs shares one 256 x 256 tile, each loading its own 128 rows
+// of X_q and its own half of the W_q rows), which halves the operand bytes each SM must pull from
+// L2 per MAC.  No cluster multicast load is used anywhere.
+//
+// The kernel is persistent (a static tile list per CTA / CTA pair), so the epilogue of tile i
+// overlaps the main loop of tile i+1.  Every wait on an mbarrier is bounded: after ~2 s the CTA
+// raises Q8_ERR_TIMEOUT in the status word, all roles leave their loops, in-flight copies are
+// drained and TMEM is released before the CTA exits.
 
 #include <cuda.h>
 
@@ -22,33 +28,39 @@ namespace q8 {
 
 namespace {
 
-constexpr int BLOCK_M = 128;      // UMMA M (cta_group::1): accumulator row i <-> TMEM lane i
-constexpr int BLOCK_K = 128;      // bytes == int8 elements per stage row: one 128-byte swizzle span
-constexpr int UMMA_K = 32;        // K of one kind::i8 instruction
-constexpr int kAccStages = 2;     // TMEM accumulator double buffering
-constexpr int kEpilogueWarps = 4; // one per TMEM lane quarter
+constexpr int BLOCK_M = 128;       // accumulator rows per CTA: row i <-> TMEM lane i
+constexpr int BLOCK_K = 128;       // bytes == int8 elements per stage row: one 128-byte swizzle span
+constexpr int UMMA_K = 32;         // K of one kind::i8 instruction
+constexpr int kAccStages = 2;      // TMEM accumulator double buffering
+constexpr int kEpilogueWarps = 8;  // two per TMEM lane quarter, each taking half of the tile's columns
 constexpr int kThreads = 64 + 32 * kEpilogueWarps;
+constexpr int kStagingBytesPerWarp = 32 * 32 * 4;  // the 32 x 32 fp32 block one tcgen05.ld hands to a warp
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
-template <int BLOCK_N>
+template <int BLOCK_N, int CTAS>
 struct Cfg {
+    static constexpr int kBRows = BLOCK_N / CTAS;  // W_q rows each CTA loads
     static constexpr int kABytes = BLOCK_M * BLOCK_K;
-    static constexpr int kBBytes = BLOCK_N * BLOCK_K;
+    static constexpr int kBBytes = kBRows * BLOCK_K;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = (192 * 1024) / kStageBytes > 8 ? 8 : (192 * 1024) / kStageBytes;
+    static constexpr int kStagingBytes = kEpilogueWarps * kStagingBytesPerWarp;
+    static constexpr int kBiasBytes = kEpilogueWarps * 32 * 4;  // b_q of the 32 columns a warp is working on
+    static constexpr int kRingBudget = 227 * 1024 - 1024 - 256 - kStagingBytes - kBiasBytes;  // left for the operand ring
+    static constexpr int kStages = kRingBudget / kStageBytes > 8 ? 8 : kRingBudget / kStageBytes;
     static constexpr int kTmemCols = kAccStages * BLOCK_N < 32 ? 32 : kAccStages * BLOCK_N;
-    static constexpr int kBiasBytes = kEpilogueWarps * BLOCK_N * 4;  // one private b_q copy per epilogue warp
     static constexpr int kBarrierBytes = (2 * kStages + 2 * kAccStages) * 8 + 16;
     // +1024: the dynamic shared window is only 16-byte aligned; tiles need 1024 (swizzle atom)
-    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBiasBytes + kBarrierBytes;
+    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kStagingBytes + kBiasBytes + kBarrierBytes;
+    static constexpr int kColsPerWarp = BLOCK_N / 2 < 32 ? 32 : BLOCK_N / 2;  // BLOCK_N = 32 leaves half the warps idle
     static_assert((kTmemCols & (kTmemCols - 1)) == 0 && kTmemCols <= 512, "TMEM columns: power of two <= 512");
-    static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "UMMA N for M = 128");
+    static_assert(BLOCK_N % 32 == 0 && BLOCK_N >= 32 && BLOCK_N <= 256, "UMMA N");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
     // Instruction descriptor of tcgen05.mma kind::i8: D = S32, A = B = signed 8-bit, both K-major.
-    static constexpr uint32_t kInstrDesc = (2u << 4)                           // D format: S32
-                                           | (1u << 7)                         // A format: signed int8
-                                           | (1u << 10)                        // B format: signed int8
-                                           | ((uint32_t)(BLOCK_N >> 3) << 17)  // N / 8
-                                           | ((uint32_t)(BLOCK_M >> 4) << 24); // M / 16
+    static constexpr uint32_t kInstrDesc = (2u << 4)                                    // D format: S32
+                                           | (1u << 7)                                  // A format: signed int8
+                                           | (1u << 10)                                 // B format: signed int8
+                                           | ((uint32_t)(BLOCK_N >> 3) << 17)           // N / 8
+                                           | ((uint32_t)((BLOCK_M * CTAS) >> 4) << 24); // M / 16
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -168,17 +180,184 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// ------------------------------------------------------------------ the kernel
-template <int BLOCK_N>
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, GemmArgs a)
+// ---- cluster / cta_group::2 forms
+__device__ __forceinline__ uint32_t cluster_ctarank()
 {
-    using C = Cfg<BLOCK_N>;
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory variable in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Load into this CTA's shared memory; completion bytes are reported to an mbarrier that may live in
+// the other CTA of the pair (no multicast: every CTA fetches exactly the bytes it stores).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int32_t c_inner,
+                                                 int32_t c_outer, uint32_t bar_cluster_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(bar_cluster_addr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrives on the mbarrier at the same shared-memory offset in both CTAs of the pair.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    const uint16_t mask = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(mask)
+        : "memory");
+}
+
+// ---- TMA store of a staged fp32 block
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t c_inner, int32_t c_outer, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(src)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// ---- GELU without erff: gelu(y) = max(y, 0) - a * Phi(-a), a = |y|, with
+// Phi(-a) = 2^p(a) and p a degree-6 fit of log2 Phi(-a) on [0, 5.6] (p(0) = -1 exactly; beyond 5.6
+// a * Phi(-a) < 1e-7 and a is clamped).  Absolute error of a * Phi(-a) below 1e-7, so the result is
+// within fp32 rounding of the erf form.  Six FMAs and one ex2 per element.
+__device__ __forceinline__ float gelu_fast(float y)
+{
+    const float a = fminf(fabsf(y), 5.6f);
+    float p = 2.9923698093625717e-05f;
+    p = fmaf(p, a, -0.0007398707093670964f);
+    p = fmaf(p, a, 0.007977453991770744f);
+    p = fmaf(p, a, -0.05323817580938339f);
+    p = fmaf(p, a, -0.45891568064689636f);
+    p = fmaf(p, a, -1.1511471271514893f);
+    p = fmaf(p, a, -1.0f);
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(p));
+    return fmaf(-a, e, fmaxf(y, 0.0f));
+}
+
+// ------------------------------------------------------------------ epilogue of one warp
+// The warp owns 32 accumulator rows (its TMEM lane quarter) x COLS columns of the tile and walks
+// them in 32-column blocks: tcgen05.ld (one row per lane) -> + b_q -> int-to-float ->
+// * 1/(S_x S_w) -> GELU -> store.  With tma_store (N % 4 == 0, Y 16-byte aligned) the 32 x 32 fp32
+// block is staged in shared memory in the 128-byte-swizzled layout of the output tensor map
+// (row = lane, 16-byte piece g at position g ^ (lane & 7): bank-conflict free) and written by one
+// TMA store, clipped at the matrix edge by the hardware; otherwise every lane stores its own row.
+// Once the last TMEM load of the tile has landed the accumulator buffer is handed back (release()).
+template <int COLS, typename Release>
+__device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
+                                              uint32_t taddr, int64_t row0, int64_t col0, const int32_t (&bqv)[COLS / 32],
+                                              float inv, uint8_t *stage, int32_t *bq_s, int lane, Release release)
+{
+    constexpr int NCHUNK = COLS / 32;
+    const int64_t row = row0 + lane;
+    const bool row_ok = row < a.M;
+#pragma unroll
+    for (int ci = 0; ci < NCHUNK; ++ci) {
+        const int64_t nb = col0 + 32 * ci;
+        // b_q of these 32 columns (one per lane, computed before the accumulator was ready) -> all lanes
+        __syncwarp();
+        bq_s[lane] = bqv[ci];
+        __syncwarp();
+        uint32_t v[32];
+        tmem_ld_32x32(taddr + (uint32_t)(32 * ci), v);
+        tmem_ld_wait();
+        if (ci + 1 == NCHUNK) release();
+        if (nb >= a.N || row0 >= a.M) continue;  // warp-uniform: the block lies outside the matrix
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+            const int4 b = *reinterpret_cast<const int4 *>(bq_s + 4 * g);
+            v[4 * g + 0] = (uint32_t)add_wrap((int32_t)v[4 * g + 0], b.x);
+            v[4 * g + 1] = (uint32_t)add_wrap((int32_t)v[4 * g + 1], b.y);
+            v[4 * g + 2] = (uint32_t)add_wrap((int32_t)v[4 * g + 2], b.z);
+            v[4 * g + 3] = (uint32_t)add_wrap((int32_t)v[4 * g + 3], b.w);
+        }
+        if (a.dbg_acc != nullptr && row_ok) {
+            int32_t *drow = a.dbg_acc + row * a.N + nb;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (nb + j < a.N) drow[j] = (int32_t)v[j];
+        }
+        if (a.act == Q8_ACT_GELU) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                v[j] = __float_as_uint(gelu_fast(__fmul_rn(__int2float_rn((int32_t)v[j]), inv)));
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__fmul_rn(__int2float_rn((int32_t)v[j]), inv));
+        }
+        if (tma_store) {
+            if (lane == 0) tma_store_wait_read();  // the previous block has left the staging buffer
+            __syncwarp();
+            uint8_t *srow = stage + lane * 128;
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+                *reinterpret_cast<uint4 *>(srow + ((g ^ (lane & 7)) << 4)) =
+                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            fence_proxy_async_smem();  // generic-proxy writes above -> visible to the TMA (async proxy)
+            __syncwarp();
+            if (lane == 0) tma_store_2d(tmap_y, (int32_t)nb, (int32_t)row0, smem_u32(stage));
+        } else if (row_ok) {
+            float *yrow = a.Y + row * a.N + nb;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (nb + j < a.N) yrow[j] = __uint_as_float(v[j]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int BLOCK_N, int CTAS>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                    const __grid_constant__ CUtensorMap tmap_y, GemmArgs a, int tma_store)
+{
+    using C = Cfg<BLOCK_N, CTAS>;
+    constexpr int TILE_M = BLOCK_M * CTAS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *smem_a = smem;
     uint8_t *smem_b = smem + C::kStages * C::kABytes;
-    int32_t *smem_bq = reinterpret_cast<int32_t *>(smem + C::kStages * C::kStageBytes);
+    uint8_t *smem_stage = smem + C::kStages * C::kStageBytes;  // multiple of 1024 from the base
+    int32_t *smem_bq = reinterpret_cast<int32_t *>(smem_stage + C::kStagingBytes);
     uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<uint8_t *>(smem_bq) + C::kBiasBytes);
     uint64_t *full_bar = bars;
     uint64_t *empty_bar = bars + C::kStages;
@@ -188,74 +367,93 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta_rank = CTAS == 2 ? cluster_ctarank() : 0u;
+    const bool leader = cta_rank == 0;
+    const int64_t unit = blockIdx.x / CTAS, num_units = gridDim.x / CTAS;  // a unit = one CTA or one CTA pair
     const int64_t tiles_n = (a.N + BLOCK_N - 1) / BLOCK_N;
-    const int64_t tiles_m = (a.M + BLOCK_M - 1) / BLOCK_M;
+    const int64_t tiles_m = (a.M + TILE_M - 1) / TILE_M;
     const int64_t num_tiles = tiles_m * tiles_n;
     const int num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; ++s) {
-            mbar_init(smem_u32(full_bar + s), 1);
-            mbar_init(smem_u32(empty_bar + s), 1);
+            mbar_init(smem_u32(full_bar + s), 1);   // the (leader's) producer arrives once, with the byte count
+            mbar_init(smem_u32(empty_bar + s), 1);  // one tcgen05.commit per use
         }
         for (int s = 0; s < kAccStages; ++s) {
             mbar_init(smem_u32(tmem_full_bar + s), 1);
-            mbar_init(smem_u32(tmem_empty_bar + s), kEpilogueWarps);
+            mbar_init(smem_u32(tmem_empty_bar + s), kEpilogueWarps * CTAS);  // every epilogue warp of the unit
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), C::kTmemCols);
+    if (warp == 1) {
+        if (CTAS == 2) tmem_alloc_pair(smem_u32(tmem_slot), C::kTmemCols);
+        else tmem_alloc(smem_u32(tmem_slot), C::kTmemCols);
+    }
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync_all();  // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer (each CTA loads its own rows) ----------------
         if (lane == 0) {
             int s = 0;
             uint32_t phase = 0;
-            int issued = 0;  // k-blocks issued so far (for the drain on abort)
+            int issued = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int32_t m0 = (int32_t)((tile / tiles_n) * BLOCK_M);
-                const int32_t n0 = (int32_t)((tile % tiles_n) * BLOCK_N);
+            for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
+                const int32_t m0 = (int32_t)((tile / tiles_n) * TILE_M + cta_rank * BLOCK_M);
+                const int32_t n0 = (int32_t)((tile % tiles_n) * BLOCK_N + cta_rank * C::kBRows);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(smem_u32(empty_bar + s), phase ^ 1u, abort_flag, a.status);
                     if (!ok) break;
                     const uint32_t fb = smem_u32(full_bar + s);
-                    mbar_expect_tx(fb, C::kStageBytes);
-                    tma_load_2d(smem_u32(smem_a + s * C::kABytes), &tmap_x, kb * BLOCK_K, m0, fb);
-                    tma_load_2d(smem_u32(smem_b + s * C::kBBytes), &tmap_w, kb * BLOCK_K, n0, fb);
+                    const uint32_t dst_a = smem_u32(smem_a + s * C::kABytes), dst_b = smem_u32(smem_b + s * C::kBBytes);
+                    if (CTAS == 1) {
+                        mbar_expect_tx(fb, C::kStageBytes);
+                        tma_load_2d(dst_a, &tmap_x, kb * BLOCK_K, m0, fb);
+                        tma_load_2d(dst_b, &tmap_w, kb * BLOCK_K, n0, fb);
+                    } else {
+                        // both CTAs report their bytes to the leader's barrier, which the MMA warp waits on
+                        if (leader) mbar_expect_tx(fb, 2 * C::kStageBytes);
+                        const uint32_t fb_leader = map_to_cta(fb, 0);
+                        tma_load_2d_pair(dst_a, &tmap_x, kb * BLOCK_K, m0, fb_leader);
+                        tma_load_2d_pair(dst_b, &tmap_w, kb * BLOCK_K, n0, fb_leader);
+                    }
                     ++issued;
                     if (++s == C::kStages) { s = 0; phase ^= 1u; }
                 }
             }
             if (!ok) {
                 // Aborting: let the copies already issued land before the CTA gives up its shared memory.
-                const int pending = issued < C::kStages ? issued : C::kStages;
-                for (int i = 0; i < pending; ++i) {
-                    const int k = issued - 1 - i;  // the i-th most recent k-block
-                    const int st = k % C::kStages;
-                    const uint32_t par = (uint32_t)((k / C::kStages) & 1);
-                    const uint64_t t0 = global_timer_ns();
-                    while (!mbar_try_wait(smem_u32(full_bar + st), par) && global_timer_ns() - t0 < 50000000ull) {}
+                const uint64_t t0 = global_timer_ns();
+                if (CTAS == 1 || leader) {
+                    const int pending = issued < C::kStages ? issued : C::kStages;
+                    for (int i = 0; i < pending; ++i) {
+                        const int k = issued - 1 - i;  // the i-th most recent k-block
+                        const uint32_t par = (uint32_t)((k / C::kStages) & 1);
+                        while (!mbar_try_wait(smem_u32(full_bar + k % C::kStages), par) &&
+                               global_timer_ns() - t0 < 50000000ull) {}
+                    }
+                } else {
+                    while (global_timer_ns() - t0 < 1000000ull) {}  // the peer cannot poll the leader's barrier
                 }
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        // ---------------- MMA issuer (the leader CTA drives the pair) ----------------
+        if (lane == 0 && leader) {
             int s = 0;
             uint32_t phase = 0;
             int as = 0;
             uint32_t aphase = 0;
-            bool ok = true;
-            bool committed = false;
+            bool ok = true, committed = false;
             int last_as = 0;
             uint32_t last_aphase = 0;
-            for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
                 ok = mbar_wait(smem_u32(tmem_empty_bar + as), aphase ^ 1u, abort_flag, a.status);
                 if (!ok) break;
                 tc_fence_after();
@@ -269,14 +467,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 #pragma unroll
                     for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                         // +32 bytes along K inside the swizzle span == +2 in the (addr >> 4) field
-                        umma_i8(tmem_d, da + (uint64_t)(k * (UMMA_K >> 4)), db + (uint64_t)(k * (UMMA_K >> 4)),
-                                C::kInstrDesc, (uint32_t)((kb | k) != 0));
+                        const uint64_t adv = (uint64_t)(k * (UMMA_K >> 4));
+                        if (CTAS == 2) umma_i8_pair(tmem_d, da + adv, db + adv, C::kInstrDesc, (uint32_t)((kb | k) != 0));
+                        else umma_i8(tmem_d, da + adv, db + adv, C::kInstrDesc, (uint32_t)((kb | k) != 0));
                     }
-                    umma_commit(smem_u32(empty_bar + s));  // frees the stage once these MMAs have read it
+                    // frees the stage (in both CTAs) once these MMAs have read it
+                    if (CTAS == 2) umma_commit_pair(smem_u32(empty_bar + s));
+                    else umma_commit(smem_u32(empty_bar + s));
                     if (++s == C::kStages) { s = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(smem_u32(tmem_full_bar + as));  // accumulator complete
+                if (CTAS == 2) umma_commit_pair(smem_u32(tmem_full_bar + as));  // accumulator complete
+                else umma_commit(smem_u32(tmem_full_bar + as));
                 committed = true;
                 last_as = as;
                 last_aphase = aphase;
@@ -291,85 +493,63 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     } else {
         // ---------------- epilogue ----------------
-        const int ew = warp - 2;            // 0 .. kEpilogueWarps-1
-        const int quarter = warp & 3;       // TMEM lanes this warp may touch: 32*quarter .. +31
+        const int ew = warp - 2;       // 0 .. 7
+        const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32*quarter .. +31
+        const int col_off = (ew >> 2) * C::kColsPerWarp;
+        const bool active = col_off < BLOCK_N;
         const float S_out = __fmul_rn(__ldg(a.S_x), __ldg(a.S_w));
         const float inv = __fdiv_rn(1.0f, S_out);
-        const bool vec_ok = ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
-        const bool dbg_vec = a.dbg_acc && ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.dbg_acc) & 15u) == 0);
+        uint8_t *stage = smem_stage + ew * kStagingBytesPerWarp;
+        int32_t *bq_s = smem_bq + ew * 32;
         int as = 0;
         uint32_t aphase = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-            const int64_t m0 = (tile / tiles_n) * BLOCK_M;
+        for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
+            const int64_t m0 = (tile / tiles_n) * TILE_M + cta_rank * BLOCK_M;
             const int64_t n0 = (tile % tiles_n) * BLOCK_N;
-            // b_q for this tile's columns (Sec. 3: bias quantised at S_x * S_w).  Each warp keeps its own
-            // copy, so the epilogue warps never have to wait for one another.
-            int32_t *bq = smem_bq + ew * BLOCK_N;
-            __syncwarp();
-            for (int c = lane; c < BLOCK_N; c += 32) {
-                const int64_t n = n0 + c;
-                bq[c] = (a.bias != nullptr && n < a.N) ? quantize_bias(__ldg(a.bias + n), S_out) : 0;
+            // b_q of this warp's columns (Sec. 3: bias quantised at S_x * S_w), fetched before the accumulator is needed
+            int32_t bqv[C::kColsPerWarp / 32];
+#pragma unroll
+            for (int ci = 0; ci < C::kColsPerWarp / 32; ++ci) {
+                const int64_t n = n0 + col_off + 32 * ci + lane;
+                bqv[ci] = (active && a.bias != nullptr && n < a.N) ? quantize_bias(__ldg(a.bias + n), S_out) : 0;
             }
-            __syncwarp();
             ok = mbar_wait(smem_u32(tmem_full_bar + as), aphase, abort_flag, a.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int64_t row = m0 + quarter * 32 + lane;
-            const bool row_ok = row < a.M;
-            float *yrow = a.Y + row * a.N;
-            int32_t *drow = a.dbg_acc ? a.dbg_acc + row * a.N : nullptr;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BLOCK_N; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + c0), r);
-                tmem_ld_wait();
-                if (n0 + c0 >= a.N) continue;  // warp-uniform
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    const int64_t n = n0 + c0 + 4 * g;
-                    int32_t v[4];
-                    float y[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        v[j] = add_wrap((int32_t)r[4 * g + j], bq[c0 + 4 * g + j]);
-                        y[j] = finish_output(v[j], inv, a.act);
-                    }
-                    if (!row_ok) continue;
-                    if (vec_ok) {
-                        if (n < a.N) *reinterpret_cast<float4 *>(yrow + n) = make_float4(y[0], y[1], y[2], y[3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            if (n + j < a.N) yrow[n + j] = y[j];
-                    }
-                    if (drow) {
-                        if (dbg_vec) {
-                            if (n < a.N) *reinterpret_cast<int4 *>(drow + n) = make_int4(v[0], v[1], v[2], v[3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                if (n + j < a.N) drow[n + j] = v[j];
-                        }
-                    }
+            // hands the accumulator buffer back to the MMA warp (called once this warp's TMEM loads are done)
+            auto release = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CTAS == 2) mbar_arrive_cluster(map_to_cta(smem_u32(tmem_empty_bar + as), 0));
+                    else mbar_arrive(smem_u32(tmem_empty_bar + as));
                 }
-            }
-            // hand the accumulator buffer back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(tmem_empty_bar + as));
+            };
+            if (active)
+                epilogue_warp<C::kColsPerWarp>(a, &tmap_y, tma_store != 0,
+                                               tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
+                                               m0 + quarter * 32, n0 + col_off, bqv, inv, stage, bq_s, lane, release);
+            else
+                release();
             if (++as == kAccStages) { as = 0; aphase ^= 1u; }
         }
+        if (lane == 0) tma_store_wait_all();
     }
 
     // ---------------- teardown (reached by every thread, also when aborting) ----------------
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) {
+        __syncwarp();
+        cluster_sync_all();  // the peer has finished with this CTA's barriers and with the shared accumulators
+    }
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, C::kTmemCols);
+        if (CTAS == 2) tmem_dealloc_pair(tmem_base, C::kTmemCols);
+        else tmem_dealloc(tmem_base, C::kTmemCols);
     }
 }
 
@@ -407,6 +587,22 @@ bool make_tmap(CUtensorMap *map, const int8_t *base, int64_t rows, int64_t K, in
     return r == CUDA_SUCCESS;
 }
 
+// Row-major fp32 output [M, N] as a tensor map of 32 x 32 boxes (128 bytes wide), 128-byte swizzle.
+// Stores that reach past row M or column N are clipped by the hardware.
+bool make_tmap_out(CUtensorMap *map, float *base, int64_t M, int64_t N)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 int sm_count()
 {
     static int n = [] {
@@ -417,43 +613,104 @@ int sm_count()
     return n;
 }
 
-template <int BLOCK_N>
+int g_force_block_n = 0, g_force_ctas = 0;  // set by q8_tune_gemm_tile(); 0 = choose automatically
+
+template <int BLOCK_N, int CTAS>
 cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
 {
-    using C = Cfg<BLOCK_N>;
+    using C = Cfg<BLOCK_N, CTAS>;
+    auto kernel = gemm_tcgen05_kernel<BLOCK_N, CTAS>;
     static bool attr_set[64] = {};  // the opt-in shared-memory size is a per-device, per-function attribute
+    static int max_units[64] = {};  // co-resident CTAs (CTAS = 1) or CTA pairs (CTAS = 2) on the device
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        e = cudaFuncSetAttribute(gemm_tcgen05_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 C::kSmemBytes);
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        int units = sm_count() / CTAS;
+        if (CTAS == 2) {
+            cudaLaunchConfig_t probe = {};
+            probe.gridDim = dim3((unsigned)(2 * units));
+            probe.blockDim = dim3(kThreads);
+            probe.dynamicSmemBytes = C::kSmemBytes;
+            cudaLaunchAttribute pattr;
+            pattr.id = cudaLaunchAttributeClusterDimension;
+            pattr.val.clusterDim.x = 2;
+            pattr.val.clusterDim.y = 1;
+            pattr.val.clusterDim.z = 1;
+            probe.attrs = &pattr;
+            probe.numAttrs = 1;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &probe) == cudaSuccess && clusters > 0 &&
+                clusters < units)
+                units = clusters;
+            (void)cudaGetLastError();
+        }
+        max_units[dev] = units;
+        attr_set[dev] = true;
     }
-    CUtensorMap tx, tw;
-    if (!make_tmap(&tx, a.Xq, a.M, a.K, BLOCK_M) || !make_tmap(&tw, a.Wq, a.N, a.K, BLOCK_N))
+    CUtensorMap tx, tw, ty;
+    if (!make_tmap(&tx, a.Xq, a.M, a.K, BLOCK_M) || !make_tmap(&tw, a.Wq, a.N, a.K, C::kBRows))
         return cudaErrorInvalidValue;
-    const int64_t tiles = ((a.M + BLOCK_M - 1) / BLOCK_M) * ((a.N + BLOCK_N - 1) / BLOCK_N);
-    const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-    gemm_tcgen05_kernel<BLOCK_N><<<grid, kThreads, C::kSmemBytes, s>>>(tx, tw, a);
+    // the TMA store needs a 16-byte aligned base and row pitch; otherwise lanes store their rows directly
+    int tma_store = ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
+    if (tma_store) {
+        if (!make_tmap_out(&ty, a.Y, a.M, a.N)) return cudaErrorInvalidValue;
+    } else {
+        ty = tx;  // never dereferenced
+    }
+    const int64_t tiles = ((a.M + BLOCK_M * CTAS - 1) / (BLOCK_M * CTAS)) * ((a.N + BLOCK_N - 1) / BLOCK_N);
+    const int units = (int)(tiles < max_units[dev] ? tiles : max_units[dev]);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(units * CTAS));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = CTAS;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kernel, tx, tw, ty, a, tma_store);
     LaunchInfo &li = last_launch_info();
     li.gemm_kernel = 1;
     li.block_n = BLOCK_N;
-    li.grid = grid;
+    li.ctas = CTAS;
+    li.grid = units * CTAS;
     li.launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
-// Relative time of one 32-deep K step of a 128 x bn tile: the tensor pipe needs bn/2 cycles, reading
-// the (128 + bn) x 32 operand bytes from shared memory needs (128 + bn)/4; plus a fixed per-step cost.
+// Relative time of one 32-deep K step of a 128 x bn tile on one SM: the tensor pipe needs bn/2 cycles,
+// reading the (128 + bn) x 32 operand bytes from shared memory needs (128 + bn)/4; plus a fixed per-step cost.
 double tile_step_cost(int bn)
 {
     const double mma = bn / 2.0, smem = (128 + bn) / 4.0;
     return (mma > smem ? mma : smem) + 8.0;
 }
 
+cudaError_t launch_by_shape(int bn, int ctas, const GemmArgs &a, cudaStream_t s)
+{
+    if (ctas == 2) return launch_cfg<256, 2>(a, s);
+    switch (bn) {
+        case 256: return launch_cfg<256, 1>(a, s);
+        case 128: return launch_cfg<128, 1>(a, s);
+        case 64: return launch_cfg<64, 1>(a, s);
+        default: return launch_cfg<32, 1>(a, s);
+    }
+}
+
 }  // namespace
+
+void set_gemm_tile_override(int block_n, int ctas)
+{
+    g_force_block_n = block_n;
+    g_force_ctas = ctas;
+}
 
 bool tcgen05_gemm_supported(const GemmArgs &a)
 {
@@ -463,9 +720,14 @@ bool tcgen05_gemm_supported(const GemmArgs &a)
 
 cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s)
 {
+    if (g_force_ctas == 2 || (g_force_ctas == 1 && g_force_block_n != 0))
+        return launch_by_shape(g_force_block_n, g_force_ctas, a, s);
     const int sms = sm_count();
+    // Large problems: CTA pairs on 256 x 256 tiles (least operand traffic per MAC) once every pair has work.
+    const int64_t pair_tiles = ((a.M + 255) / 256) * ((a.N + 255) / 256);
+    if (a.N >= 192 && a.M > 128 && pair_tiles >= sms / 2) return launch_by_shape(256, 2, a, s);
+    // Otherwise single-CTA tiles: pick the width that minimises (waves over the SMs) x (time of one tile).
     const int64_t tm = (a.M + BLOCK_M - 1) / BLOCK_M;
-    // Pick the tile width that minimises (waves over the SMs) x (time of one tile).
     int best = 32;
     double best_cost = 0.0;
     for (int bn : {256, 128, 64, 32}) {
@@ -477,12 +739,7 @@ cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s)
             best_cost = cost;
         }
     }
-    switch (best) {
-        case 256: return launch_cfg<256>(a, s);
-        case 128: return launch_cfg<128>(a, s);
-        case 64: return launch_cfg<64>(a, s);
-        default: return launch_cfg<32>(a, s);
-    }
+    return launch_by_shape(best, 1, a, s);
 }
 
 }  // namespace q8

@@ -43,6 +43,7 @@ struct LaunchInfo {
     int gemm_kernel = 0;  // 0 none, 1 tcgen05, 2 generic
     int launches = 0;
     int block_n = 0;
+    int ctas = 0;  // CTAs cooperating on one tile (1, or 2 for cta_group::2)
     int grid = 0;
 };
 LaunchInfo &last_launch_info();
@@ -60,6 +61,7 @@ cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, co
 
 // ---- GEMM launchers ----
 bool tcgen05_gemm_supported(const GemmArgs &a);
+void set_gemm_tile_override(int block_n, int ctas);  // 0, 0 = automatic choice
 cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s);  // q8_gemm_sm100.cu
 cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_generic.cu
 
