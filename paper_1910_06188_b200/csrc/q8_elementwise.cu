@@ -193,8 +193,9 @@ __device__ __forceinline__ float4 dequant4(uint32_t w, float inv)
     return f;
 }
 
-// VEC: one thread moves 4 table bytes (one 4-byte load) to one 16-byte store; consecutive lanes
-// cover consecutive pieces of a row, so a warp reads 128 and writes 512 contiguous bytes.
+// VEC: a CTA walks token rows (four at a time, so four independent gathers are in flight per thread);
+// within a row one thread moves 4 table bytes (one 4-byte load) to one 16-byte streaming store, so a
+// warp reads 128 and writes 512 contiguous bytes.  No per-element index arithmetic beyond adds.
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads) embedding_kernel(const int32_t *__restrict__ ids, int64_t T,
                                                              const int8_t *__restrict__ Eq,
@@ -203,24 +204,33 @@ __global__ void __launch_bounds__(kThreads) embedding_kernel(const int32_t *__re
                                                              int32_t *__restrict__ status)
 {
     const float inv = __fdiv_rn(1.0f, __ldg(S_e));
-    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
     if (VEC) {
-        const int64_t per_row = H >> 2;
-        const int64_t total = T * per_row;
-        for (int64_t w = tid; w < total; w += nthreads) {
-            const int64_t t = w / per_row, c = w - t * per_row;
-            const int64_t id = __ldg(ids + t);
-            uint32_t q = 0u;
-            if (id >= 0 && id < V) {
-                q = __ldg(reinterpret_cast<const uint32_t *>(Eq + id * H) + c);
-            } else if (c == 0 && status) {
-                atomicOr(status, 1 << Q8_ERR_INDEX);
+        const int per_row = (int)(H >> 2);
+        for (int64_t t0 = (int64_t)blockIdx.x * 4; t0 < T; t0 += (int64_t)gridDim.x * 4) {
+            int64_t id[4];
+            bool ok[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                id[r] = (t0 + r < T) ? (int64_t)__ldg(ids + t0 + r) : -1;
+                ok[r] = id[r] >= 0 && id[r] < V;
+                if (!ok[r] && t0 + r < T && threadIdx.x == 0 && status) atomicOr(status, 1 << Q8_ERR_INDEX);
             }
-            __stcs(reinterpret_cast<float4 *>(out) + w, dequant4(q, inv));
-            if (rows_q) reinterpret_cast<uint32_t *>(rows_q)[w] = q;
+            for (int c = threadIdx.x; c < per_row; c += blockDim.x) {
+                uint32_t q[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    q[r] = ok[r] ? __ldg(reinterpret_cast<const uint32_t *>(Eq + id[r] * H) + c) : 0u;
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    if (t0 + r >= T) break;
+                    __stcs(reinterpret_cast<float4 *>(out + (t0 + r) * H) + c, dequant4(q[r], inv));
+                    if (rows_q) reinterpret_cast<uint32_t *>(rows_q + (t0 + r) * H)[c] = q[r];
+                }
+            }
         }
     } else {
+        const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
         const int64_t total = T * H;
         for (int64_t e = tid; e < total; e += nthreads) {
             const int64_t t = e / H, h = e - t * H;
@@ -281,8 +291,10 @@ cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, co
     if (T <= 0 || H <= 0) return cudaSuccess;
     const bool vec = (H % 4 == 0) && aligned16(Eq) && aligned16(out) && (rows_q == nullptr || aligned16(rows_q));
     if (vec) {
-        embedding_kernel<true><<<grid_for(T * (H >> 2), kThreads * 2, 8), kThreads, 0, s>>>(ids, T, Eq, S_e, V, H, out,
-                                                                                      rows_q, status);
+        // one thread per 4-byte piece of a row, rounded up to whole warps; a CTA takes 4 rows per iteration
+        int threads = (int)(((H >> 2) + 31) / 32 * 32);
+        if (threads > kThreads) threads = kThreads;
+        embedding_kernel<true><<<grid_for((T + 3) / 4, 1, 16), threads, 0, s>>>(ids, T, Eq, S_e, V, H, out, rows_q, status);
     } else {
         embedding_kernel<false><<<grid_for(T * H, kThreads, 8), kThreads, 0, s>>>(ids, T, Eq, S_e, V, H, out,
                                                                                  rows_q, status);
