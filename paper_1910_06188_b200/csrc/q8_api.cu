@@ -69,15 +69,15 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
                       int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic)
 {
     last_launch_info() = LaunchInfo();
-    if (!X || !Wq || !S_w || !Y || !workspace) return Q8_ERR_NULL;
     q8_status st = check_gemm_shape(M, N, K);
     if (st != Q8_OK) return st;
+    if (M == 0 || N == 0) return Q8_OK;  // nothing to compute; empty tensors may carry NULL pointers
+    if (!X || !Wq || !S_w || !Y || !workspace) return Q8_ERR_NULL;
     if (act != Q8_ACT_NONE && act != Q8_ACT_GELU) return Q8_ERR_ARG;
     if (!aligned_to(X, 4) || !aligned_to(Y, 4) || !aligned_to(S_w, 4) || (S_x && !aligned_to(S_x, 4)) ||
         (bias && !aligned_to(bias, 4)) || (dbg_acc && !aligned_to(dbg_acc, 4)) || !aligned_to(workspace, 256))
         return Q8_ERR_ALIGN;
     if (workspace_bytes < q8_linear_workspace_bytes(M, N, K)) return Q8_ERR_WORKSPACE;
-    if (M == 0 || N == 0) return Q8_OK;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WorkspaceHeader *hdr = static_cast<WorkspaceHeader *>(workspace);
@@ -194,14 +194,14 @@ q8_status q8_linear_q(const int8_t *Xq, const float *S_x, const int8_t *Wq, cons
                       void *stream)
 {
     last_launch_info() = LaunchInfo();
-    if (!Xq || !S_x || !Wq || !S_w || !Y) return Q8_ERR_NULL;
     q8_status st = check_gemm_shape(M, N, K);
     if (st != Q8_OK) return st;
+    if (M == 0 || N == 0) return Q8_OK;
+    if (!Xq || !S_x || !Wq || !S_w || !Y) return Q8_ERR_NULL;
     if (act != Q8_ACT_NONE && act != Q8_ACT_GELU) return Q8_ERR_ARG;
     if (!aligned_to(Y, 4) || !aligned_to(S_w, 4) || !aligned_to(S_x, 4) || (bias && !aligned_to(bias, 4)) ||
         (dbg_acc && !aligned_to(dbg_acc, 4)) || (dev_status && !aligned_to(dev_status, 4)))
         return Q8_ERR_ALIGN;
-    if (M == 0 || N == 0) return Q8_OK;
     GemmArgs g;
     g.Xq = Xq;
     g.Wq = Wq;

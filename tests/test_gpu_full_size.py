@@ -1,0 +1,107 @@
+"""Parity at the benchmark's full size and launch configuration: the BERT-Large FC set at
+M = 24576 tokens with static scales, automatic tile choice (CTA pairs on 256 x 256 tiles).
+
+The oracle cannot run 0.6 tera-ops in seconds, so: the quantised activation is compared in full;
+three row slabs (first rows, rows straddling a tile boundary in the middle, last rows) are compared
+with the oracle on exactly those rows (rows are independent once the scale is fixed); random single
+entries are checked one by one; and the whole Int32 matrix is compared with the generic CUDA-core
+kernel as a secondary, on-device check."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import q8_oracle as o
+from paper_1910_06188_b200 import binding as q8
+from paper_1910_06188_b200 import synth
+from tests.gpu_util import REL_TOL, dev
+
+pytestmark = pytest.mark.gpu
+
+M = synth.BERT_LARGE["batch"] * synth.BERT_LARGE["seq"]
+LAYERS = synth.fc_set(synth.BERT_LARGE["hidden"], synth.BERT_LARGE["ffn"])
+
+
+@pytest.mark.parametrize("name,K,N,act", LAYERS)
+def test_bert_large_fc_full_size(name, K, N, act):
+    idx = [n for n, *_ in LAYERS].index(name)
+    X = synth.activation(M, K, synth.seed_for(4, 10 * idx))
+    calib = synth.activation(4096, K, synth.seed_for(4, 10 * idx + 1))
+    W = synth.weight(N, K, synth.seed_for(4, 10 * idx + 2))
+    b = synth.bias(N, synth.seed_for(4, 10 * idx + 3))
+
+    state = q8.new_calibrate_state()
+    q8.q8_calibrate(dev(calib), 0.9999, state)
+    S_x_dev = q8.calibrate_S_x(state).clone()
+    S_x = o.EmaState().update(o.absmax(calib), 0.9999)
+    assert S_x_dev.item() == S_x
+    Wq, S_w = q8.q8_quantize_weight(dev(W))
+    Wq_ref, S_w_ref, _ = o.quantize_weight(W)
+    assert np.array_equal(Wq.cpu().numpy(), Wq_ref) and S_w.item() == S_w_ref
+
+    Xd, bd = dev(X), dev(b)
+    xq = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    ws = q8.new_workspace(M, N, K)
+    Y = q8.q8_linear(Xd, Wq, S_w, S_x_dev, bd, act, workspace=ws, dbg_Xq=xq, dbg_acc=acc)
+    info = q8.q8_last_launch_info()
+    assert q8.q8_poll_status(ws) == (q8.Q8_OK, 0)
+    assert info["gemm_kernel"] == 1 and info["ctas"] == 2 and info["block_n"] == 256  # what bench.py times
+
+    # (1) the whole quantised activation
+    xq_ref = o.quantize(X, S_x)
+    assert np.array_equal(xq.cpu().numpy(), xq_ref)
+
+    # (2) row slabs against the oracle on the same rows
+    mid = (M // 2 // 256) * 256
+    for lo, hi in [(0, 48), (mid - 24, mid + 24), (M - 40, M)]:
+        ref = o.linear(X[lo:hi], Wq_ref, S_w_ref, S_x, b, act)
+        assert np.array_equal(acc[lo:hi].cpu().numpy(), ref["acc"]), f"{name}: Int32 rows {lo}:{hi}"
+        err = np.abs(Y[lo:hi].cpu().numpy().astype(np.float64) - ref["y"]).max()
+        assert err <= REL_TOL * np.abs(ref["y"]).max(), f"{name}: rows {lo}:{hi} err {err}"
+
+    # (3) random single entries, one by one
+    rng = np.random.default_rng(1234 + idx)
+    ms = rng.integers(0, M, size=200)
+    ns = rng.integers(0, N, size=200)
+    bq = o.quantize_bias(b, S_x, S_w_ref)
+    got = acc[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].cpu().numpy()
+    for m, n, g in zip(ms, ns, got):
+        assert o.linear_entry(xq_ref[m], Wq_ref[n], int(bq[n])) == g, f"{name}: entry ({m},{n})"
+
+    # (4) the whole Int32 matrix against the generic kernel (secondary, on-device)
+    acc2 = torch.empty_like(acc)
+    Y2 = q8.q8_linear_generic(Xd, Wq, S_w, S_x_dev, bd, act, workspace=ws, dbg_acc=acc2)
+    assert q8.q8_last_launch_info()["gemm_kernel"] == 2
+    assert torch.equal(acc, acc2)
+    assert (Y - Y2).abs().max().item() <= REL_TOL * Y2.abs().max().item()
+
+
+@pytest.mark.parametrize("block_n,ctas", [(32, 1), (64, 1), (128, 1), (256, 1), (256, 2)])
+def test_every_tile_shape_matches_the_oracle(block_n, ctas):
+    """Each instantiation of the tcgen05 kernel, forced through the tuning hook, on ragged shapes."""
+    from tests.gpu_util import check_linear
+    try:
+        q8.q8_tune_gemm_tile(block_n, ctas)
+        for (Mm, Nn, Kk, act) in [(300, 200, 400, 1), (1000, 520, 272, 0), (515, 1030, 144, 1)]:
+            X = synth.activation(Mm, Kk, seed=1100 + Mm)
+            W = synth.weight(Nn, Kk, seed=1101 + Mm)
+            bb = synth.bias(Nn, seed=1102 + Mm)
+            info = check_linear(X, W, bb, act=act)
+            assert (info["block_n"], info["ctas"]) == (block_n, ctas)
+    finally:
+        q8.q8_tune_gemm_tile(0, 0)
+    with pytest.raises(q8.Q8Error):
+        q8.q8_tune_gemm_tile(48, 1)
+
+
+def test_empty_problem_is_a_noop():
+    Wq = torch.ones((8, 16), dtype=torch.int8, device="cuda")
+    S = torch.ones(1, device="cuda")
+    X = torch.empty((0, 16), device="cuda")
+    Y = q8.q8_linear(X, Wq, S, S, None, 0)
+    assert Y.shape == (0, 8)
+    assert q8.q8_last_launch_info()["launches"] == 0
+    xq, _ = q8.q8_quantize_activation(torch.empty(0, device="cuda"), S)
+    assert xq.numel() == 0
+    out = q8.q8_embedding(torch.empty(0, dtype=torch.int32, device="cuda"), Wq, S)
+    assert out.shape == (0, 16)
