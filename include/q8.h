@@ -115,6 +115,29 @@ q8_status q8_linear_generic(const float *X, const int8_t *Wq, const float *S_w, 
                             void *workspace, size_t workspace_bytes, int8_t *dbg_Xq,
                             int32_t *dbg_acc, void *stream);
 
+/* q8_linear for callers that cannot allocate device memory.  (The paper has no counterpart: this is
+ * a deployment convenience, not part of the method.)
+ * Intended for code that runs where cudaMalloc is off limits: a serving loop whose memory was
+ * partitioned at start-up, a plugin working inside an engine that owns all allocations, a process
+ * whose allocator is frozen after initialisation.  It computes exactly what q8_linear computes, with
+ * the same arguments minus the workspace: the scratch (status word + Int8 activation) is a fixed
+ * array inside the library image, present on every GPU that loads the library until the process
+ * exits.  The call itself performs no allocation of any kind.
+ *   Limit: M * K <= Q8_NOALLOC_MAX_MK (16 Mi elements, i.e. 16 MiB of scratch + a 256-byte header);
+ *     larger activations are refused with Q8_ERR_WORKSPACE before anything is launched.
+ *   status_word (host pointer, may be NULL) receives the device address of the status word, which
+ *     can be handed to q8_poll_status.
+ *   The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   Every call on a device uses the same array: calls that may overlap on the GPU (different
+ *     streams without ordering, or host threads) race on it.  Order them, or use q8_linear with
+ *     separate workspaces.  The header words are cleared at the start of each call; the rest is
+ *     simply overwritten. */
+#define Q8_NOALLOC_MAX_MK (16 * 1024 * 1024)
+q8_status q8_linear_noalloc(const float *X, const int8_t *Wq, const float *S_w, const float *S_x,
+                            const float *bias, int act, float *Y, int64_t M, int64_t N, int64_t K,
+                            int8_t *dbg_Xq, int32_t *dbg_acc, void **status_word, void *stream);
+
 /* Quantised embedding layer in inference mode (Sec. 3): gathers Int8 rows of the table and hands
  * them to the FP32 consumer dequantised: out[t, :] = Eq[ids[t], :] / S_e.
  *   ids [T] int32; Eq [V,H] int8; S_e 1 fp32; out [T,H] fp32 (written); rows_q [T,H] int8 optional

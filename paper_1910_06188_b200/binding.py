@@ -32,6 +32,7 @@ SIGNATURES = {
     "q8_linear_workspace_bytes": (_sz, [_i64, _i64, _i64]),
     "q8_linear_q": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "q8_linear_generic": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
+    "q8_linear_noalloc": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _vp, C.POINTER(_vp), _vp]),
     "q8_embedding": (_int, [_vp, _i64, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _vp]),
     "q8_poll_status": (_int, [_vp, C.POINTER(C.c_uint32), _vp]),
     "q8_status_string": (C.c_char_p, [_int]),
@@ -206,6 +207,37 @@ def q8_linear_q(Xq, S_x, Wq, S_w, bias=None, act: int = Q8_ACT_NONE, Y=None, dbg
                             _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "q8_linear_q")
     return Y
+
+
+Q8_NOALLOC_MAX_MK = 16 * 1024 * 1024
+
+
+def q8_linear_noalloc(X, Wq, S_w, S_x=None, bias=None, act: int = Q8_ACT_NONE, Y=None, dbg_Xq=None, dbg_acc=None,
+                      stream=None):
+    """q8_linear without a caller workspace: for callers that may not allocate device memory (the scratch
+    is a fixed array inside the library, M*K <= Q8_NOALLOC_MAX_MK).  Y must be supplied by such callers;
+    when it is None this binding allocates it with torch for convenience.  Returns (Y, status_word_address)."""
+    M, K = X.shape
+    N, K2 = Wq.shape
+    if K != K2:
+        raise ValueError(f"X is [M,{K}] but Wq is [N,{K2}]")
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float32, device=X.device)
+    word = C.c_void_p(0)
+    st = load().q8_linear_noalloc(_ptr(X, torch.float32, "X"), _ptr(Wq, torch.int8, "Wq"),
+                                  _ptr(S_w, torch.float32, "S_w"), _ptr(S_x, torch.float32, "S_x"),
+                                  _ptr(bias, torch.float32, "bias"), int(act), _ptr(Y, torch.float32, "Y"), M, N, K,
+                                  _ptr(dbg_Xq, torch.int8, "dbg_Xq"), _ptr(dbg_acc, torch.int32, "dbg_acc"),
+                                  C.byref(word), _stream(stream))
+    _check(st, "q8_linear_noalloc")
+    return Y, word.value
+
+
+def q8_poll_status_at(address: int, stream=None) -> Tuple[int, int]:
+    """q8_poll_status on a raw device address (e.g. the status word returned by q8_linear_noalloc)."""
+    raw = C.c_uint32(0)
+    st = load().q8_poll_status(C.c_void_p(address), C.byref(raw), _stream(stream))
+    return int(st), int(raw.value)
 
 
 def q8_embedding(ids, Eq, S_e, out=None, rows_q=None, dev_status=None, stream=None) -> torch.Tensor:

@@ -64,6 +64,8 @@ q8_status run_gemm(const GemmArgs &g, bool force_generic, cudaStream_t s)
     return Q8_OK;
 }
 
+}  // namespace
+
 q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
                       float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
                       int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic)
@@ -104,7 +106,7 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
     return run_gemm(g, force_generic, s);
 }
 
-}  // namespace
+
 }  // namespace q8
 
 using namespace q8;

@@ -65,6 +65,11 @@ void set_gemm_tile_override(int block_n, int ctas);  // 0, 0 = automatic choice
 cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s);  // q8_gemm_sm100.cu
 cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_generic.cu
 
+// The body of q8_linear / q8_linear_generic: validates, quantises X into `workspace`, runs the GEMM (q8_api.cu).
+q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
+                      float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
+                      int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic);
+
 // ---- epilogue arithmetic shared by both GEMM kernels ----
 // Bias quantised at the product scale: Clamp(nint(b * S_out), -(2^31-1), 2^31-1).
 __device__ __forceinline__ int32_t quantize_bias(float b, float S_out)
