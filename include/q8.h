@@ -146,6 +146,21 @@ q8_status q8_linear_noalloc(const float *X, const int8_t *Wq, const float *S_w, 
 q8_status q8_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,
                        int64_t H, float *out, int8_t *rows_q, int32_t *dev_status, void *stream);
 
+/* FP32 support operations of the BERT encoder.  Sec. 3 keeps Softmax, Layer Normalization and GELU
+ * in FP32, and the attention score / context products are not FC layers, so they are not quantised;
+ * these two calls let a whole encoder forward run through this library.
+ *
+ * out[r, :] = LayerNorm(x[r, :] + r1[r, :] + r2[r, :]) * gamma + beta   (rows x H, row-major fp32;
+ * r1, r2, gamma, beta may be NULL: no residual / gamma 1 / beta 0; mean and variance over H, biased
+ * variance, eps inside the square root).  H <= 12288.  out may alias x, r1 or r2. */
+q8_status q8_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma,
+                           const float *beta, float eps, int64_t rows, int64_t H, float *out, void *stream);
+
+/* Multi-head self-attention without mask, head dimension 64, fp32:
+ *   qkv [B*S, 3*H] = [q | k | v] per token (H = heads * 64), ctx [B*S, H] (written):
+ *   ctx[b, i, h*64 : h*64+64] = sum_j softmax_j(q_i . k_j / 8) v_j  over the S tokens of sequence b. */
+q8_status q8_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, void *stream);
+
 /* Synchronises `stream`, reads the device status word at `dev_status` (a q8_linear workspace
  * pointer works: the word sits at offset 0), clears it, and returns the lowest-numbered code
  * whose bit was set (Q8_OK if none).  `raw_bits` (host pointer, may be NULL) receives the word. */

@@ -222,3 +222,69 @@ int64_t q8o_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, float S_e
     }
     return bad;
 }
+
+/* ---- FP32-kept encoder operations (Sec. 3: Softmax and Layer Normalization stay in floating point;
+ * the encoder is the BERT of Devlin et al.).  Evaluated in fp64, straight from the definitions. ---- */
+
+/* out[r][:] = LayerNorm(x[r][:] + r1[r][:] + r2[r][:]) * gamma + beta; r1, r2, gamma, beta may be NULL.
+ * Mean and (biased) variance over the H features of a row, eps inside the square root. */
+void q8o_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma, const float *beta,
+                       double eps, int64_t rows, int64_t H, double *out)
+{
+    for (int64_t r = 0; r < rows; ++r) {
+        double mean = 0.0, var = 0.0;
+        for (int64_t h = 0; h < H; ++h) {
+            double v = (double)x[r * H + h];
+            if (r1) v += (double)r1[r * H + h];
+            if (r2) v += (double)r2[r * H + h];
+            out[r * H + h] = v;
+            mean += v;
+        }
+        mean /= (double)H;
+        for (int64_t h = 0; h < H; ++h) {
+            double d = out[r * H + h] - mean;
+            var += d * d;
+        }
+        var /= (double)H;
+        double rstd = 1.0 / sqrt(var + eps);
+        for (int64_t h = 0; h < H; ++h) {
+            double g = gamma ? (double)gamma[h] : 1.0, b = beta ? (double)beta[h] : 0.0;
+            out[r * H + h] = (out[r * H + h] - mean) * rstd * g + b;
+        }
+    }
+}
+
+/* Multi-head self-attention without mask: qkv [B*S][3*heads*d] = [q | k | v] per token,
+ * ctx[b][i][h] = sum_j softmax_j(q_i . k_j / sqrt(d)) v_j. */
+void q8o_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, int64_t d, double *ctx)
+{
+    int64_t H = heads * d, P = 3 * H;
+    double scale = 1.0 / sqrt((double)d);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t b = 0; b < B; ++b) {
+        for (int64_t hd = 0; hd < heads; ++hd) {
+            double *score = (double *)malloc((size_t)S * sizeof(double));
+            for (int64_t i = 0; i < S; ++i) {
+                const float *q = qkv + (b * S + i) * P + hd * d;
+                double mx = -INFINITY, sum = 0.0;
+                for (int64_t j = 0; j < S; ++j) {
+                    const float *k = qkv + (b * S + j) * P + H + hd * d;
+                    double s = 0.0;
+                    for (int64_t t = 0; t < d; ++t) s += (double)q[t] * (double)k[t];
+                    score[j] = s * scale;
+                    if (score[j] > mx) mx = score[j];
+                }
+                for (int64_t j = 0; j < S; ++j) {
+                    score[j] = exp(score[j] - mx);
+                    sum += score[j];
+                }
+                for (int64_t t = 0; t < d; ++t) {
+                    double acc = 0.0;
+                    for (int64_t j = 0; j < S; ++j) acc += score[j] * (double)qkv[(b * S + j) * P + 2 * H + hd * d + t];
+                    ctx[(b * S + i) * H + hd * d + t] = acc / sum;
+                }
+            }
+            free(score);
+        }
+    }
+}

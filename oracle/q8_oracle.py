@@ -63,6 +63,10 @@ def lib() -> C.CDLL:
         L.q8o_linear_entry.argtypes = [i8p, i8p, C.c_int64, C.c_int32]
         L.q8o_embedding.restype = C.c_int64
         L.q8o_embedding.argtypes = [i32p, C.c_int64, i8p, C.c_float, C.c_int64, C.c_int64, i8p, dp]
+        L.q8o_add_layernorm.restype = None
+        L.q8o_add_layernorm.argtypes = [fp, fp, fp, fp, fp, C.c_double, C.c_int64, C.c_int64, dp]
+        L.q8o_attention.restype = None
+        L.q8o_attention.argtypes = [fp, C.c_int64, C.c_int64, C.c_int64, C.c_int64, dp]
         _lib = L
     return _lib
 
@@ -207,3 +211,25 @@ def embedding(ids, Eq, S_e):
     bad = lib().q8o_embedding(_p(ids, C.c_int32), T, _p(Eq, C.c_int8), C.c_float(float(np.float32(S_e))),
                               V, H, _p(rows, C.c_int8), _p(out, C.c_double))
     return rows, out, int(bad)
+
+
+def add_layernorm(x, r1=None, r2=None, gamma=None, beta=None, eps: float = 1e-12) -> np.ndarray:
+    """fp64 LayerNorm(x + r1 + r2) * gamma + beta over the last dimension."""
+    x = _f32(x)
+    rows, H = x.shape
+    opt = lambda a: _f32(a) if a is not None else None
+    r1, r2, gamma, beta = opt(r1), opt(r2), opt(gamma), opt(beta)
+    out = np.empty((rows, H), np.float64)
+    pf = lambda a: _p(a, C.c_float) if a is not None else None
+    lib().q8o_add_layernorm(_p(x, C.c_float), pf(r1), pf(r2), pf(gamma), pf(beta), float(eps), rows, H,
+                            _p(out, C.c_double))
+    return out
+
+
+def attention(qkv, B: int, S: int, heads: int, d: int = 64) -> np.ndarray:
+    """fp64 multi-head self-attention on the fused projection [B*S, 3*heads*d]; returns ctx [B*S, heads*d]."""
+    qkv = _f32(qkv)
+    assert qkv.shape == (B * S, 3 * heads * d)
+    ctx = np.empty((B * S, heads * d), np.float64)
+    lib().q8o_attention(_p(qkv, C.c_float), B, S, heads, d, _p(ctx, C.c_double))
+    return ctx

@@ -5,4 +5,4 @@ The arithmetic runs in hand-written CUDA kernels behind a C-ABI shared library
 first use and loading fails loudly when it has not been built: there is no CPU fallback.
 """
 
-__all__ = ["binding", "synth", "build"]
+__all__ = ["binding", "synth", "build", "encoder"]

@@ -34,6 +34,8 @@ SIGNATURES = {
     "q8_linear_generic": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
     "q8_linear_noalloc": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _vp, C.POINTER(_vp), _vp]),
     "q8_embedding": (_int, [_vp, _i64, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "q8_add_layernorm": (_int, [_vp, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp]),
+    "q8_attention": (_int, [_vp, _i64, _i64, _i64, _vp, _vp]),
     "q8_poll_status": (_int, [_vp, C.POINTER(C.c_uint32), _vp]),
     "q8_status_string": (C.c_char_p, [_int]),
     "q8_last_launch_info": (None, [C.POINTER(_int)] * 5),
@@ -251,6 +253,32 @@ def q8_embedding(ids, Eq, S_e, out=None, rows_q=None, dev_status=None, stream=No
                              _stream(stream))
     _check(st, "q8_embedding")
     return out
+
+
+def q8_add_layernorm(x, r1=None, r2=None, gamma=None, beta=None, eps: float = 1e-12, out=None, stream=None):
+    """out = LayerNorm(x + r1 + r2) * gamma + beta over the last dimension (fp32, Sec. 3)."""
+    rows, H = x.shape
+    if out is None:
+        out = torch.empty_like(x)
+    st = load().q8_add_layernorm(_ptr(x, torch.float32, "x"), _ptr(r1, torch.float32, "r1"),
+                                 _ptr(r2, torch.float32, "r2"), _ptr(gamma, torch.float32, "gamma"),
+                                 _ptr(beta, torch.float32, "beta"), float(eps), rows, H,
+                                 _ptr(out, torch.float32, "out"), _stream(stream))
+    _check(st, "q8_add_layernorm")
+    return out
+
+
+def q8_attention(qkv, B: int, S: int, heads: int, ctx=None, stream=None):
+    """fp32 multi-head self-attention (head dimension 64, no mask) on the fused projection [B*S, 3*heads*64]."""
+    H = heads * 64
+    if tuple(qkv.shape) != (B * S, 3 * H):
+        raise ValueError(f"qkv must be [{B * S}, {3 * H}], got {tuple(qkv.shape)}")
+    if ctx is None:
+        ctx = torch.empty((B * S, H), dtype=torch.float32, device=qkv.device)
+    st = load().q8_attention(_ptr(qkv, torch.float32, "qkv"), B, S, heads, _ptr(ctx, torch.float32, "ctx"),
+                             _stream(stream))
+    _check(st, "q8_attention")
+    return ctx
 
 
 def q8_poll_status(dev_status: torch.Tensor, stream=None) -> Tuple[int, int]:

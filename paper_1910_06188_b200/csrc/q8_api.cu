@@ -238,6 +238,34 @@ q8_status q8_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const fl
     return Q8_OK;
 }
 
+q8_status q8_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma, const float *beta,
+                           float eps, int64_t rows, int64_t H, float *out, void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (rows < 0 || H < 0 || H > 12288 || rows > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
+    if (rows == 0 || H == 0) return Q8_OK;
+    if (!x || !out) return Q8_ERR_NULL;
+    if (!(eps >= 0.0f)) return Q8_ERR_ARG;
+    if (!aligned_to(x, 4) || !aligned_to(out, 4) || !aligned_to(r1, 4) || !aligned_to(r2, 4) || !aligned_to(gamma, 4) ||
+        !aligned_to(beta, 4))
+        return Q8_ERR_ALIGN;
+    Q8_CUDA_TRY(launch_add_layernorm(x, r1, r2, gamma, beta, eps, rows, H, out, static_cast<cudaStream_t>(stream)));
+    last_launch_info().launches = 1;
+    return Q8_OK;
+}
+
+q8_status q8_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (B < 0 || S < 0 || heads < 0 || B > 65535 || heads > 65535 || S > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
+    if (B == 0 || S == 0 || heads == 0) return Q8_OK;
+    if (!qkv || !ctx) return Q8_ERR_NULL;
+    if (!aligned_to(qkv, 8) || !aligned_to(ctx, 8)) return Q8_ERR_ALIGN;  // 8-byte vector accesses per row of 64
+    Q8_CUDA_TRY(launch_attention(qkv, B, S, heads, ctx, static_cast<cudaStream_t>(stream)));
+    last_launch_info().launches = 1;
+    return Q8_OK;
+}
+
 q8_status q8_poll_status(void *dev_status, uint32_t *raw_bits, void *stream)
 {
     if (!dev_status) return Q8_ERR_NULL;

@@ -59,6 +59,11 @@ cudaError_t launch_ema_update(CalibState *st, float decay, cudaStream_t s);
 cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,
                              int64_t H, float *out, int8_t *rows_q, int32_t *status, cudaStream_t s);
 
+// ---- fp32 encoder support (q8_support.cu) ----
+cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma,
+                                 const float *beta, float eps, int64_t rows, int64_t H, float *out, cudaStream_t s);
+cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, cudaStream_t s);
+
 // ---- GEMM launchers ----
 bool tcgen05_gemm_supported(const GemmArgs &a);
 void set_gemm_tile_override(int block_n, int ctas);  // 0, 0 = automatic choice

@@ -1,0 +1,217 @@
+// FP32 operations of the BERT encoder that Q8BERT leaves unquantised (Sec. 3: Softmax, Layer
+// Normalization and GELU stay in FP32; the attention score / context products are not FC layers):
+// residual add + LayerNorm, and scaled-dot-product self-attention.  They exist so that a whole
+// encoder forward can run through this library; the quantised path proper is in the other files.
+
+#include <math.h>
+
+#include "q8_internal.cuh"
+
+namespace q8 {
+
+namespace {
+
+// ------------------------------------------------------------------ out = LayerNorm(x + r1 + r2) * gamma + beta
+// One CTA per row.  The summed row is kept in shared memory, so the inputs are read once; mean and
+// variance are the two-pass forms (sum, then sum of squared deviations), reduced through warp shuffles.
+constexpr int kLnThreads = 256;
+
+__device__ __forceinline__ float block_sum(float v, float *scratch)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();  // scratch may still be read from the previous reduction
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float t = 0.0f;
+#pragma unroll
+    for (int w = 0; w < kLnThreads / 32; ++w) t += scratch[w];
+    return t;
+}
+
+__global__ void __launch_bounds__(kLnThreads) add_layernorm_kernel(const float *__restrict__ x,
+                                                                   const float *__restrict__ r1,
+                                                                   const float *__restrict__ r2,
+                                                                   const float *__restrict__ gamma,
+                                                                   const float *__restrict__ beta, float eps, int64_t H,
+                                                                   float *__restrict__ out)
+{
+    extern __shared__ float row[];
+    __shared__ float scratch[kLnThreads / 32];
+    const int64_t base = (int64_t)blockIdx.x * H;
+    float s = 0.0f;
+    for (int64_t h = threadIdx.x; h < H; h += kLnThreads) {
+        float v = x[base + h];
+        if (r1) v += r1[base + h];
+        if (r2) v += r2[base + h];
+        row[h] = v;
+        s += v;
+    }
+    const float mean = block_sum(s, scratch) / (float)H;
+    float q = 0.0f;
+    for (int64_t h = threadIdx.x; h < H; h += kLnThreads) {
+        const float d = row[h] - mean;
+        q += d * d;
+    }
+    const float var = block_sum(q, scratch) / (float)H;
+    const float rstd = 1.0f / sqrtf(var + eps);
+    for (int64_t h = threadIdx.x; h < H; h += kLnThreads) {
+        const float g = gamma ? gamma[h] : 1.0f, b = beta ? beta[h] : 0.0f;
+        out[base + h] = (row[h] - mean) * rstd * g + b;
+    }
+}
+
+// ------------------------------------------------------------------ self-attention, head dimension 64, no mask
+// ctx[b, i, head] = softmax_j(q_i . k_j / 8) v_j with q, k, v read from the fused projection
+// qkv[T, 3H] = [q | k | v].  One CTA per (64 queries, head, sequence); keys and values stream through
+// shared memory in tiles of 64 with the running-max / running-sum form of softmax, all in fp32.
+// Thread (ty, tx) of the 16 x 16 CTA owns rows {2ty, 2ty+1, 2ty+32, 2ty+33} x columns {2tx, 2tx+1, 2tx+32,
+// 2tx+33} of the 64 x 64 score tile and of the output tile, so its operands are two 8-byte loads each and
+// consecutive lanes touch consecutive banks.  Q, K and P are held transposed with a pitch of 66 floats.
+constexpr int kD = 64, kTile = 64, kPitch = 66;
+constexpr int kAttnSmemBytes = (3 * kD * kPitch + kTile * kD) * (int)sizeof(float);
+
+__device__ __forceinline__ int own_index(int t, int a) { return 2 * t + (a & 1) + 32 * (a >> 1); }
+
+__global__ void __launch_bounds__(256) attention_kernel(const float *__restrict__ qkv, int64_t S, int64_t H,
+                                                        float scale, float *__restrict__ ctx)
+{
+    extern __shared__ __align__(16) float attn_smem[];
+    float(*Qt)[kPitch] = reinterpret_cast<float(*)[kPitch]>(attn_smem);                    // Qt[d][i]
+    float(*Kt)[kPitch] = reinterpret_cast<float(*)[kPitch]>(attn_smem + kD * kPitch);       // Kt[d][j]
+    float(*Pt)[kPitch] = reinterpret_cast<float(*)[kPitch]>(attn_smem + 2 * kD * kPitch);   // Pt[j][i]
+    float(*Vs)[kD] = reinterpret_cast<float(*)[kD]>(attn_smem + 3 * kD * kPitch);           // Vs[j][d]
+
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int64_t q0 = (int64_t)blockIdx.x * kTile, head = blockIdx.y, seq = blockIdx.z;
+    const int64_t row_pitch = 3 * H;
+    const float *base = qkv + seq * S * row_pitch + head * kD;
+
+    // queries of this CTA (pre-scaled), transposed; rows past the sequence end are zero
+    for (int e = threadIdx.x; e < kTile * kD; e += 256) {
+        const int i = e / kD, d = e % kD;
+        Qt[d][i] = (q0 + i < S) ? base[(q0 + i) * row_pitch + d] * scale : 0.0f;
+    }
+
+    float o[4][4] = {};
+    float m[4], l[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        m[a] = -INFINITY;
+        l[a] = 0.0f;
+    }
+
+    for (int64_t j0 = 0; j0 < S; j0 += kTile) {
+        __syncthreads();  // previous tile fully consumed (and Qt written, on the first pass)
+        for (int e = threadIdx.x; e < kTile * kD; e += 256) {
+            const int j = e / kD, d = e % kD;
+            const bool ok = j0 + j < S;
+            Kt[d][j] = ok ? base[(j0 + j) * row_pitch + H + d] : 0.0f;
+            Vs[j][d] = ok ? base[(j0 + j) * row_pitch + 2 * H + d] : 0.0f;
+        }
+        __syncthreads();
+
+        float s[4][4] = {};
+#pragma unroll 8
+        for (int d = 0; d < kD; ++d) {
+            const float2 q01 = *reinterpret_cast<const float2 *>(&Qt[d][2 * ty]);
+            const float2 q23 = *reinterpret_cast<const float2 *>(&Qt[d][2 * ty + 32]);
+            const float2 k01 = *reinterpret_cast<const float2 *>(&Kt[d][2 * tx]);
+            const float2 k23 = *reinterpret_cast<const float2 *>(&Kt[d][2 * tx + 32]);
+            const float qv[4] = {q01.x, q01.y, q23.x, q23.y}, kv[4] = {k01.x, k01.y, k23.x, k23.y};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) s[a][b] = fmaf(qv[a], kv[b], s[a][b]);
+        }
+        // keys past the sequence end do not take part
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+            if (j0 + own_index(tx, b) >= S) {
+#pragma unroll
+                for (int a = 0; a < 4; ++a) s[a][b] = -INFINITY;
+            }
+        // running max / sum per query row (a row's 64 scores live in the 16 threads that share ty)
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            float mx = fmaxf(fmaxf(s[a][0], s[a][1]), fmaxf(s[a][2], s[a][3]));
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+            const float m_new = fmaxf(m[a], mx);
+            const float corr = expf(m[a] - m_new);  // exp(-inf) = 0 on the first tile
+            float sum = 0.0f;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                s[a][b] = expf(s[a][b] - m_new);
+                sum += s[a][b];
+            }
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+            l[a] = l[a] * corr + sum;
+            m[a] = m_new;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) o[a][b] *= corr;
+        }
+        // probabilities to shared memory (transposed), then O += P V
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int j = own_index(tx, b);
+            *reinterpret_cast<float2 *>(&Pt[j][2 * ty]) = make_float2(s[0][b], s[1][b]);
+            *reinterpret_cast<float2 *>(&Pt[j][2 * ty + 32]) = make_float2(s[2][b], s[3][b]);
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int j = 0; j < kTile; ++j) {
+            const float2 p01 = *reinterpret_cast<const float2 *>(&Pt[j][2 * ty]);
+            const float2 p23 = *reinterpret_cast<const float2 *>(&Pt[j][2 * ty + 32]);
+            const float2 v01 = *reinterpret_cast<const float2 *>(&Vs[j][2 * tx]);
+            const float2 v23 = *reinterpret_cast<const float2 *>(&Vs[j][2 * tx + 32]);
+            const float pv[4] = {p01.x, p01.y, p23.x, p23.y}, vv[4] = {v01.x, v01.y, v23.x, v23.y};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) o[a][b] = fmaf(pv[a], vv[b], o[a][b]);
+        }
+    }
+
+    float *obase = ctx + seq * S * H + head * kD;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int64_t i = q0 + own_index(ty, a);
+        if (i >= S) continue;
+        const float inv = 1.0f / l[a];
+        *reinterpret_cast<float2 *>(obase + i * H + 2 * tx) = make_float2(o[a][0] * inv, o[a][1] * inv);
+        *reinterpret_cast<float2 *>(obase + i * H + 2 * tx + 32) = make_float2(o[a][2] * inv, o[a][3] * inv);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma,
+                                 const float *beta, float eps, int64_t rows, int64_t H, float *out, cudaStream_t s)
+{
+    if (rows <= 0 || H <= 0) return cudaSuccess;
+    add_layernorm_kernel<<<(unsigned)rows, kLnThreads, (size_t)H * sizeof(float), s>>>(x, r1, r2, gamma, beta, eps, H,
+                                                                                       out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, cudaStream_t s)
+{
+    if (B <= 0 || S <= 0 || heads <= 0) return cudaSuccess;
+    static bool attr_set[64] = {};  // opt-in shared-memory size: per device, per function
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    dim3 grid((unsigned)((S + kTile - 1) / kTile), (unsigned)heads, (unsigned)B);
+    attention_kernel<<<grid, 256, kAttnSmemBytes, s>>>(qkv, S, heads * kD, 1.0f / 8.0f, ctx);
+    return cudaGetLastError();
+}
+
+}  // namespace q8

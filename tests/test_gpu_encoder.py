@@ -1,0 +1,166 @@
+"""Encoder-level checks: the FP32 support kernels against the oracle, and whole encoder forwards.
+
+A forward chains ~50-100 quantised layers, and layer k+1 quantises what layer k computed in fp32,
+so an ulp of difference upstream can flip a nearest-integer decision downstream.  Bit-exactness is
+therefore checked per call with the call's own input: for every q8_linear inside the forward the CPU
+oracle is given the same fp32 input bytes that the layer received (and its own quantisation of the
+seeded weights) and must reproduce the Int8 activation, the Int32 accumulator and the fp32 output of
+that call.  On top of that a small model is run end to end in the oracle from the seeded inputs alone."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import q8_oracle as o
+from paper_1910_06188_b200 import binding as q8
+from paper_1910_06188_b200 import encoder as enc_mod
+from paper_1910_06188_b200 import synth
+from tests.gpu_util import REL_TOL, assert_close_fp, dev
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ support kernels
+@pytest.mark.parametrize("rows,H", [(1, 4), (37, 96), (300, 768), (64, 1024), (5, 1000)])
+def test_add_layernorm(rows, H):
+    x = synth.activation(rows, H, 3000 + H)
+    r1 = synth.activation(rows, H, 3001 + H)
+    r2 = synth.normal((rows, H), 0.5, 3002 + H)
+    g = synth.normal((H,), 1.0, 3003 + H)
+    b = synth.normal((H,), 1.0, 3004 + H)
+    assert_close_fp(q8.q8_add_layernorm(dev(x), dev(r1), dev(r2), dev(g), dev(b)).cpu().numpy(),
+                    o.add_layernorm(x, r1, r2, g, b), "LN(x+r1+r2)")
+    assert_close_fp(q8.q8_add_layernorm(dev(x), dev(r1)).cpu().numpy(), o.add_layernorm(x, r1), "LN(x+r1)")
+    assert_close_fp(q8.q8_add_layernorm(dev(x)).cpu().numpy(), o.add_layernorm(x), "LN(x)")
+    xd = dev(x)
+    q8.q8_add_layernorm(xd, dev(r1), out=xd)                       # in place
+    assert_close_fp(xd.cpu().numpy(), o.add_layernorm(x, r1), "LN in place")
+
+
+@pytest.mark.parametrize("B,S,heads", [(1, 1, 1), (2, 9, 3), (3, 64, 2), (2, 70, 2), (2, 128, 12), (1, 384, 4)])
+def test_attention(B, S, heads):
+    qkv = synth.normal((B * S, 3 * heads * 64), 1.0, 3100 + S)
+    got = q8.q8_attention(dev(qkv), B, S, heads).cpu().numpy()
+    assert_close_fp(got, o.attention(qkv, B, S, heads), "attention")
+
+
+def test_attention_large_logits_stay_finite():
+    B, S, heads = 1, 130, 1
+    qkv = synth.normal((B * S, 3 * 64), 6.0, 3150)             # logits of several hundred
+    got = q8.q8_attention(dev(qkv), B, S, heads).cpu().numpy()
+    assert np.isfinite(got).all()
+    # fp32 logits of magnitude ~500 carry an absolute rounding error of ~500 * 2^-24 = 3e-5, which the
+    # exponential turns into the same relative error of the weights: bound the output error accordingly
+    ref = o.attention(qkv, B, S, heads)
+    assert np.abs(got - ref).max() <= 1e-4 * np.abs(ref).max()
+
+
+# ------------------------------------------------------------------ whole forwards
+def _oracle_weights(enc):
+    w = {}
+    for name, t in enc.fp32.items():
+        if name.startswith("b."):
+            w[name] = t
+        else:
+            w[name] = o.quantize_weight(t)[:2]        # (W_q, S_w) from the seeded fp32 tensor
+    return w
+
+
+def _teacher_forced_hook(enc, w, T, slabs, record):
+    """Checks each quantised FC of a forward against the oracle on the rows in `slabs`."""
+    def hook(l, name, X, Y, p, S_x, Xq, acc):
+        Wq_ref, S_w_ref = w[f"W.{l}.{name}"]
+        b = w[f"b.{l}.{name}"]
+        assert p["S_w"].item() == S_w_ref
+        sx = np.float32(S_x.item())
+        for lo, hi in slabs:
+            Xs = X[lo:hi].cpu().numpy()
+            ref = o.linear(Xs, Wq_ref, S_w_ref, sx, b, p["act"])
+            assert np.array_equal(Xq[lo:hi].cpu().numpy(), ref["xq"]), f"layer {l} {name}: X_q rows {lo}:{hi}"
+            assert np.array_equal(acc[lo:hi].cpu().numpy(), ref["acc"]), f"layer {l} {name}: Int32 rows {lo}:{hi}"
+            err = np.abs(Y[lo:hi].cpu().numpy() - ref["y"]).max()
+            assert err <= REL_TOL * max(np.abs(ref["y"]).max(), 1e-30), f"layer {l} {name}: fp32 rows {lo}:{hi}"
+        record.append((l, name, float(sx)))
+    return hook
+
+
+def _oracle_forward(enc, w, ids, B, S):
+    """The same forward, every step in the oracle, from the seeded inputs alone (dynamic scales)."""
+    f32 = lambda a: np.asarray(a, dtype=np.float32)
+    T = B * S
+    pos = np.tile(np.arange(S, dtype=np.int32), B)
+    typ = np.zeros(T, np.int32)
+    ew = o.embedding(ids, *w["word"])[1]
+    ep = o.embedding(pos, *w["pos"])[1]
+    et = o.embedding(typ, *w["typ"])[1]
+    h = f32(o.add_layernorm(f32(ew), f32(ep), f32(et), eps=enc_mod.LN_EPS))
+    lin = lambda l, name, X, act: f32(o.linear(X, *w[f"W.{l}.{name}"], None, w[f"b.{l}.{name}"], act)["y"])
+    for l in range(enc.L):
+        qkv = lin(l, "qkv", h, 0)
+        ctx = f32(o.attention(qkv, B, S, enc.heads))
+        ao = lin(l, "attn_out", ctx, 0)
+        h1 = f32(o.add_layernorm(ao, h, eps=enc_mod.LN_EPS))
+        f = lin(l, "ffn1", h1, 1)
+        f2 = lin(l, "ffn2", f, 0)
+        h = f32(o.add_layernorm(f2, h1, eps=enc_mod.LN_EPS))
+    return h
+
+
+def test_small_encoder_teacher_forced_and_end_to_end():
+    dims = dict(hidden=128, ffn=512, heads=2, layers=3, vocab=500, max_pos=96)
+    B, S = 3, 70
+    enc = enc_mod.Q8BertEncoder(dims, config=30, keep_fp32=True)
+    w = _oracle_weights(enc)
+    ids_h = synth.token_ids(B * S, dims["vocab"], synth.seed_for(30, 90))
+    ids = torch.from_numpy(ids_h).cuda()
+    rec = []
+    out = enc.forward(ids, B, S, scales="dynamic", debug=True,
+                      hook=_teacher_forced_hook(enc, w, B * S, [(0, B * S)], rec)).cpu().numpy()
+    assert len(rec) == 4 * dims["layers"] and enc.poll() == ((q8.Q8_OK, 0), (q8.Q8_OK, 0))
+    want = _oracle_forward(enc, w, ids_h, B, S)
+    # end to end a nearest-integer flip may occur somewhere; outputs are LayerNorm-ed (unit scale)
+    diff = np.abs(out - want)
+    assert diff.max() < 5e-2 and np.median(diff) < 1e-4, (diff.max(), np.median(diff))
+
+
+def _run_model_case(dims, config, B, S, scales, calib_batches, layers=None):
+    enc = enc_mod.Q8BertEncoder(dims, config=config, keep_fp32=True, layers=layers)
+    w = _oracle_weights(enc)
+    T = B * S
+    V = dims["vocab"]
+    if scales == "static":
+        refs = {}
+        for c in range(calib_batches):
+            cid = torch.from_numpy(synth.token_ids(T, V, synth.seed_for(config, 300 + c))).cuda()
+
+            def cal_hook(l, name, X, Y, p, S_x, Xq, acc):
+                if l == 0:                      # follow the EMA of the first layer's four quantisers in the oracle
+                    refs.setdefault(name, o.EmaState()).update(o.absmax(X.cpu().numpy()), 0.9999)
+            enc.forward(cid, B, S, scales="calibrate", decay=0.9999, hook=cal_hook)
+        for name, st in refs.items():
+            got = q8.calibrate_S_x(enc.layers[0][name]["state"]).item()
+            assert np.float32(got) == st.S_x, f"Eq. 4 scale of layer 0 {name}"
+            assert enc.layers[0][name]["state"][2].item() == calib_batches
+    ids = enc_mod.random_ids(T, V, config)
+    mid = (T // 2 // 256) * 256
+    slabs = [(0, 24), (mid - 12, mid + 12), (T - 24, T)]
+    rec = []
+    out = enc.forward(ids, B, S, scales=scales, debug=True, hook=_teacher_forced_hook(enc, w, T, slabs, rec))
+    assert len(rec) == 4 * enc.L
+    assert enc.poll() == ((q8.Q8_OK, 0), (q8.Q8_OK, 0))
+    o_np = out.cpu().numpy()
+    assert np.isfinite(o_np).all()
+    assert np.allclose(o_np.mean(1), 0, atol=1e-4) and np.allclose(o_np.var(1), 1, atol=1e-3)   # LayerNorm-ed rows
+    # int8 weights are a quarter of the fp32 bytes
+    fp32_bytes = 4 * sum(t.size for n, t in enc.fp32.items() if not n.startswith("b."))
+    assert enc.memory_bytes_int8() * 4 == fp32_bytes
+
+
+def test_bert_base_encoder_forward():
+    """BERT-Base encoder, batch 32 x seq 128: int8 embeddings, all FC layers quantised, static scales from
+    one seeded calibration batch."""
+    _run_model_case(synth.BERT_BASE, config=3, B=32, S=128, scales="static", calib_batches=1)
+
+
+def test_bert_large_encoder_forward():
+    """BERT-Large encoder, batch 64 x seq 384, EMA scales (decay 0.9999) over 16 seeded batches."""
+    _run_model_case(synth.BERT_LARGE, config=5, B=64, S=384, scales="static", calib_batches=16)

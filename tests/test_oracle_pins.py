@@ -287,3 +287,49 @@ def test_embedding_gather_and_bound():
     ids[3], ids[7] = -1, V
     rows, out, bad = o.embedding(ids, Eq, S_e)
     assert bad == 2 and not rows[3].any() and not out[7].any()
+
+
+# ---------------------------------------------------------------- FP32-kept encoder operations (Sec. 3)
+def test_layernorm_hand_example_and_moments():
+    # x = [1,2,3,4]: mean 2.5, biased variance 1.25 -> (x - 2.5) / sqrt(1.25)
+    x = np.array([[1.0, 2.0, 3.0, 4.0]], np.float32)
+    want = (np.array([1.0, 2.0, 3.0, 4.0]) - 2.5) / math.sqrt(1.25)
+    assert np.allclose(o.add_layernorm(x, eps=0.0), want, rtol=0, atol=1e-15)
+    rng = np.random.default_rng(51)
+    x = rng.standard_normal((7, 96)).astype(np.float32) * 3 + 1
+    r1 = rng.standard_normal((7, 96)).astype(np.float32)
+    g = rng.standard_normal(96).astype(np.float32)
+    b = rng.standard_normal(96).astype(np.float32)
+    y = o.add_layernorm(x, r1)
+    assert np.allclose(y.mean(1), 0, atol=1e-12) and np.allclose(y.var(1), 1, atol=1e-9)
+    z = o.add_layernorm(x, r1, None, g, b)
+    assert np.allclose(z, y * g.astype(np.float64) + b.astype(np.float64), atol=1e-12)
+    # the residual really is added before normalising
+    assert np.allclose(o.add_layernorm(x, r1), o.add_layernorm((x.astype(np.float64) + r1).astype(np.float32)), atol=1e-5)
+    assert not np.allclose(o.add_layernorm(x, r1), o.add_layernorm(x))
+
+
+def test_attention_special_cases_and_numpy():
+    rng = np.random.default_rng(53)
+    B, S, heads, d = 2, 9, 3, 64
+    H = heads * d
+    qkv = rng.standard_normal((B * S, 3 * H)).astype(np.float32)
+    got = o.attention(qkv, B, S, heads)
+    # independent numpy evaluation of softmax(q k^T / sqrt d) v
+    q = qkv[:, :H].reshape(B, S, heads, d).astype(np.float64)
+    k = qkv[:, H:2 * H].reshape(B, S, heads, d).astype(np.float64)
+    v = qkv[:, 2 * H:].reshape(B, S, heads, d).astype(np.float64)
+    sc = np.einsum("bihd,bjhd->bhij", q, k) / 8.0
+    p = np.exp(sc - sc.max(-1, keepdims=True))
+    p /= p.sum(-1, keepdims=True)
+    want = np.einsum("bhij,bjhd->bihd", p, v).reshape(B * S, H)
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
+    # identical keys -> uniform weights -> every output is the mean value of its sequence and head
+    same = qkv.copy()
+    same[:, H:2 * H] = same[0, H:2 * H]
+    got = o.attention(same, B, S, heads)
+    vmean = same[:, 2 * H:].reshape(B, S, H).astype(np.float64).mean(1)
+    assert np.allclose(got.reshape(B, S, H), vmean[:, None, :], atol=1e-12)
+    # a single token attends to itself only
+    one = rng.standard_normal((3, 3 * H)).astype(np.float32)
+    assert np.allclose(o.attention(one, 3, 1, heads), one[:, 2 * H:], atol=0)
