@@ -387,6 +387,15 @@ def run_ours(args):
             "sample": f"first {rows} of {M} token rows of each of the 4 FC layers, once ({dt:.1f} s)",
         }
 
+    # ---- whole encoder forwards (tokens/s): int8 embeddings, every FC quantised, attention / LayerNorm in fp32
+    encoder = None
+    if world == 1 and not args.no_encoder:
+        for L in layers:
+            L.clear()
+        del host_in, host_out, host_emb, emb_out
+        torch.cuda.empty_cache()
+        encoder = measure_encoders(args, torch, q8)
+
     line = {
         "metric": "q8_linear_int8_tops", "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -403,11 +412,74 @@ def run_ours(args):
         "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline,
         "cpu_baseline": cpu_baseline,
+        "encoder": encoder,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
     return 0
+
+
+def measure_encoders(args, torch, q8):
+    """Tokens/s of whole BERT-Base (32 x 128) and BERT-Large (64 x 384) encoder forwards with static scales,
+    plus where the time goes (CUDA events around every call of one extra forward)."""
+    from paper_1910_06188_b200 import encoder as enc_mod
+
+    out = {}
+    for name, dims, cfg in (("bert_base_32x128", synth.BERT_BASE, 3), ("bert_large_64x384", synth.BERT_LARGE, 5)):
+        B, S = dims["batch"], dims["seq"]
+        T = B * S
+        enc = enc_mod.Q8BertEncoder(dims, config=cfg)
+        ids = enc_mod.random_ids(T, dims["vocab"], cfg)
+        enc.forward(ids, B, S, scales="calibrate")
+        for _ in range(3):
+            enc.forward(ids, B, S)
+        torch.cuda.synchronize()
+        reps = args.encoder_steps
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            enc.forward(ids, B, S)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        codes = enc.poll()
+        # breakdown: time the three kinds of calls of one forward
+        shares = {"q8_linear": 0.0, "attention_fp32": 0.0, "layernorm_embedding": 0.0}
+        orig = {k: getattr(q8, k) for k in ("q8_linear", "q8_attention", "q8_add_layernorm", "q8_embedding")}
+        evs = []
+
+        def timed(fn, key):
+            def wrapper(*a, **k):
+                a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a0.record()
+                r = fn(*a, **k)
+                a1.record()
+                evs.append((key, a0, a1))
+                return r
+            return wrapper
+        try:
+            q8.q8_linear = timed(orig["q8_linear"], "q8_linear")
+            q8.q8_attention = timed(orig["q8_attention"], "attention_fp32")
+            q8.q8_add_layernorm = timed(orig["q8_add_layernorm"], "layernorm_embedding")
+            q8.q8_embedding = timed(orig["q8_embedding"], "layernorm_embedding")
+            enc.forward(ids, B, S)
+            torch.cuda.synchronize()
+        finally:
+            for k, fn in orig.items():
+                setattr(q8, k, fn)
+        for key, a0, a1 in evs:
+            shares[key] += a0.elapsed_time(a1)
+        fc_ops = enc.L * sum(2.0 * T * N * K for _, K, N, _ in synth.fc_set(enc.H, enc.F))
+        out[name] = {
+            "tokens_per_s": T / (ms * 1e-3), "ms_per_forward": ms, "layers": enc.L, "tokens": T,
+            "gpu_launches_per_forward": enc.launches_per_forward(), "status": [list(c) for c in codes],
+            "ms_by_kind": shares, "q8_linear_tops_inside_forward": fc_ops / (shares["q8_linear"] * 1e-3) / 1e12,
+            "int8_parameter_bytes": enc.memory_bytes_int8(),
+        }
+        del enc
+        torch.cuda.empty_cache()
+    return out
 
 
 def main():
@@ -421,6 +493,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=2048, help="token rows per layer for the cpu_baseline sample")
     ap.add_argument("--reference-rows", type=int, default=256, help="token rows per layer per step for --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-encoder", action="store_true", help="skip the whole-encoder tokens/s measurement")
+    ap.add_argument("--encoder-steps", type=int, default=5)
     ap.add_argument("--layers", default="", help="comma list of FC layers to keep (qkv,attn_out,ffn1,ffn2); default all")
     ap.add_argument("--profile-mode", action="store_true",
                     help="only warm-up + timed steps (no per-kernel pass, e2e or CPU baseline): for ncu captures")
