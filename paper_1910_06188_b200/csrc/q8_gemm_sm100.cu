@@ -504,16 +504,27 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         int as = 0;
         uint32_t aphase = 0;
         bool ok = true;
+        // The bias values of a tile are fetched one tile ahead: under the operand traffic of the main loop a
+        // global load takes microseconds, which would otherwise be exposed at the start of every tile.
+        constexpr int NCH = C::kColsPerWarp / 32;
+        float bias_next[NCH];
+        auto fetch_bias = [&](int64_t tile, float (&dst)[NCH]) {
+            const int64_t n0 = (tile % tiles_n) * BLOCK_N;
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                const int64_t n = n0 + col_off + 32 * ci + lane;
+                dst[ci] = (active && a.bias != nullptr && tile < num_tiles && n < a.N) ? __ldg(a.bias + n) : 0.0f;
+            }
+        };
+        fetch_bias(unit, bias_next);
         for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
             const int64_t m0 = (tile / tiles_n) * TILE_M + cta_rank * BLOCK_M;
             const int64_t n0 = (tile % tiles_n) * BLOCK_N;
-            // b_q of this warp's columns (Sec. 3: bias quantised at S_x * S_w), fetched before the accumulator is needed
-            int32_t bqv[C::kColsPerWarp / 32];
+            // b_q of this warp's columns (Sec. 3: bias quantised at S_x * S_w)
+            int32_t bqv[NCH];
 #pragma unroll
-            for (int ci = 0; ci < C::kColsPerWarp / 32; ++ci) {
-                const int64_t n = n0 + col_off + 32 * ci + lane;
-                bqv[ci] = (active && a.bias != nullptr && n < a.N) ? quantize_bias(__ldg(a.bias + n), S_out) : 0;
-            }
+            for (int ci = 0; ci < NCH; ++ci) bqv[ci] = quantize_bias(bias_next[ci], S_out);
+            fetch_bias(tile + num_units, bias_next);
             ok = mbar_wait(smem_u32(tmem_full_bar + as), aphase, abort_flag, a.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
