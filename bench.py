@@ -443,6 +443,16 @@ def measure_encoders(args, torch, q8):
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / reps
+        # the same forward with every quantiser fused into its producer (bit-identical result)
+        for _ in range(2):
+            enc.forward_fused(ids, B, S)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            enc.forward_fused(ids, B, S)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_fused = e0.elapsed_time(e1) / reps
         codes = enc.poll()
         # breakdown: time the three kinds of calls of one forward
         shares = {"q8_linear": 0.0, "attention_fp32": 0.0, "layernorm_embedding": 0.0}
@@ -473,7 +483,10 @@ def measure_encoders(args, torch, q8):
         fc_ops = enc.L * sum(2.0 * T * N * K for _, K, N, _ in synth.fc_set(enc.H, enc.F))
         out[name] = {
             "tokens_per_s": T / (ms * 1e-3), "ms_per_forward": ms, "layers": enc.L, "tokens": T,
-            "gpu_launches_per_forward": enc.launches_per_forward(), "status": [list(c) for c in codes],
+            "tokens_per_s_fused_requant": T / (ms_fused * 1e-3), "ms_per_forward_fused_requant": ms_fused,
+            "gpu_launches_per_forward": enc.launches_per_forward(),
+            "gpu_launches_per_forward_fused_requant": enc.launches_per_forward(fused=True),
+            "status": [list(c) for c in codes],
             "ms_by_kind": shares, "q8_linear_tops_inside_forward": fc_ops / (shares["q8_linear"] * 1e-3) / 1e12,
             "int8_parameter_bytes": enc.memory_bytes_int8(),
         }

@@ -161,6 +161,25 @@ q8_status q8_add_layernorm(const float *x, const float *r1, const float *r2, con
  *   ctx[b, i, h*64 : h*64+64] = sum_j softmax_j(q_i . k_j / 8) v_j  over the S tokens of sequence b. */
 q8_status q8_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, void *stream);
 
+/* Fused re-quantisation (Sec. 3 inference mode chained layer to layer; Eq. 1 with the consumer's Eq. 4
+ * scale): the producer of an activation also emits it as Int8 at the NEXT quantised layer's static
+ * scale S_y / S_q, so that layer can run q8_linear_q with no separate quantise pass and, for FFN1, no
+ * fp32 round trip through HBM.  The Int8 values equal Quantize(y | S) of the very fp32 value the plain
+ * call would have stored.  The fp32 output pointer (Y / out / ctx) may be NULL when only Int8 is wanted.
+ * Other arguments are as in q8_linear, q8_linear_q, q8_add_layernorm and q8_attention. */
+q8_status q8_linear_requant(const float *X, const int8_t *Wq, const float *S_w, const float *S_x,
+                            const float *bias, int act, const float *S_y, int8_t *Yq, float *Y, int64_t M,
+                            int64_t N, int64_t K, void *workspace, size_t workspace_bytes, int8_t *dbg_Xq,
+                            int32_t *dbg_acc, void *stream);
+q8_status q8_linear_q_requant(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w,
+                              const float *bias, int act, const float *S_y, int8_t *Yq, float *Y, int64_t M,
+                              int64_t N, int64_t K, int32_t *dbg_acc, int32_t *dev_status, void *stream);
+q8_status q8_add_layernorm_quant(const float *x, const float *r1, const float *r2, const float *gamma,
+                                 const float *beta, float eps, int64_t rows, int64_t H, float *out,
+                                 const float *S_q, int8_t *out_q, void *stream);
+q8_status q8_attention_quant(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx,
+                             const float *S_q, int8_t *ctx_q, void *stream);
+
 /* Synchronises `stream`, reads the device status word at `dev_status` (a q8_linear workspace
  * pointer works: the word sits at offset 0), clears it, and returns the lowest-numbered code
  * whose bit was set (Q8_OK if none).  `raw_bits` (host pointer, may be NULL) receives the word. */

@@ -36,6 +36,10 @@ SIGNATURES = {
     "q8_embedding": (_int, [_vp, _i64, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _vp]),
     "q8_add_layernorm": (_int, [_vp, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp]),
     "q8_attention": (_int, [_vp, _i64, _i64, _i64, _vp, _vp]),
+    "q8_linear_requant": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
+    "q8_linear_q_requant": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "q8_add_layernorm_quant": (_int, [_vp, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "q8_attention_quant": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "q8_poll_status": (_int, [_vp, C.POINTER(C.c_uint32), _vp]),
     "q8_status_string": (C.c_char_p, [_int]),
     "q8_last_launch_info": (None, [C.POINTER(_int)] * 5),
@@ -279,6 +283,67 @@ def q8_attention(qkv, B: int, S: int, heads: int, ctx=None, stream=None):
                              _stream(stream))
     _check(st, "q8_attention")
     return ctx
+
+
+def q8_linear_requant(X, Wq, S_w, S_x, bias, act, S_y, Yq=None, Y=None, workspace=None, dbg_Xq=None, dbg_acc=None,
+                      stream=None):
+    """q8_linear whose output is (also) emitted as Int8 at the next layer's scale S_y.  Returns Yq."""
+    M, K = X.shape
+    N = Wq.shape[0]
+    if Yq is None:
+        Yq = torch.empty((M, N), dtype=torch.int8, device=X.device)
+    if workspace is None:
+        workspace = new_workspace(M, N, K, X.device)
+    st = load().q8_linear_requant(_ptr(X, torch.float32, "X"), _ptr(Wq, torch.int8, "Wq"),
+                                  _ptr(S_w, torch.float32, "S_w"), _ptr(S_x, torch.float32, "S_x"),
+                                  _ptr(bias, torch.float32, "bias"), int(act), _ptr(S_y, torch.float32, "S_y"),
+                                  _ptr(Yq, torch.int8, "Yq"), _ptr(Y, torch.float32, "Y"), M, N, K,
+                                  _any_ptr(workspace, "workspace"), workspace.numel() * workspace.element_size(),
+                                  _ptr(dbg_Xq, torch.int8, "dbg_Xq"), _ptr(dbg_acc, torch.int32, "dbg_acc"),
+                                  _stream(stream))
+    _check(st, "q8_linear_requant")
+    return Yq
+
+
+def q8_linear_q_requant(Xq, S_x, Wq, S_w, bias, act, S_y, Yq=None, Y=None, dbg_acc=None, dev_status=None, stream=None):
+    """q8_linear_q whose output is (also) emitted as Int8 at the next layer's scale S_y.  Returns Yq."""
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    if Yq is None:
+        Yq = torch.empty((M, N), dtype=torch.int8, device=Xq.device)
+    st = load().q8_linear_q_requant(_ptr(Xq, torch.int8, "Xq"), _ptr(S_x, torch.float32, "S_x"),
+                                    _ptr(Wq, torch.int8, "Wq"), _ptr(S_w, torch.float32, "S_w"),
+                                    _ptr(bias, torch.float32, "bias"), int(act), _ptr(S_y, torch.float32, "S_y"),
+                                    _ptr(Yq, torch.int8, "Yq"), _ptr(Y, torch.float32, "Y"), M, N, K,
+                                    _ptr(dbg_acc, torch.int32, "dbg_acc"), _ptr(dev_status, torch.int32, "dev_status"),
+                                    _stream(stream))
+    _check(st, "q8_linear_q_requant")
+    return Yq
+
+
+def q8_add_layernorm_quant(x, r1, r2, S_q, out_q=None, out=None, gamma=None, beta=None, eps: float = 1e-12, stream=None):
+    """LayerNorm(x + r1 + r2) written as fp32 (`out`, optional) and as Int8 at scale S_q (`out_q`)."""
+    rows, H = x.shape
+    if out_q is None:
+        out_q = torch.empty((rows, H), dtype=torch.int8, device=x.device)
+    st = load().q8_add_layernorm_quant(_ptr(x, torch.float32, "x"), _ptr(r1, torch.float32, "r1"),
+                                       _ptr(r2, torch.float32, "r2"), _ptr(gamma, torch.float32, "gamma"),
+                                       _ptr(beta, torch.float32, "beta"), float(eps), rows, H,
+                                       _ptr(out, torch.float32, "out"), _ptr(S_q, torch.float32, "S_q"),
+                                       _ptr(out_q, torch.int8, "out_q"), _stream(stream))
+    _check(st, "q8_add_layernorm_quant")
+    return out_q
+
+
+def q8_attention_quant(qkv, B: int, S: int, heads: int, S_q, ctx_q=None, ctx=None, stream=None):
+    """fp32 self-attention whose context is (also) emitted as Int8 at scale S_q."""
+    H = heads * 64
+    if ctx_q is None:
+        ctx_q = torch.empty((B * S, H), dtype=torch.int8, device=qkv.device)
+    st = load().q8_attention_quant(_ptr(qkv, torch.float32, "qkv"), B, S, heads, _ptr(ctx, torch.float32, "ctx"),
+                                   _ptr(S_q, torch.float32, "S_q"), _ptr(ctx_q, torch.int8, "ctx_q"), _stream(stream))
+    _check(st, "q8_attention_quant")
+    return ctx_q
 
 
 def q8_poll_status(dev_status: torch.Tensor, stream=None) -> Tuple[int, int]:

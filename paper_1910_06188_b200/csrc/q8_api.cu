@@ -68,13 +68,17 @@ q8_status run_gemm(const GemmArgs &g, bool force_generic, cudaStream_t s)
 
 q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
                       float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
-                      int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic)
+                      int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic, int8_t *Yq,
+                      const float *S_y)
 {
     last_launch_info() = LaunchInfo();
     q8_status st = check_gemm_shape(M, N, K);
     if (st != Q8_OK) return st;
     if (M == 0 || N == 0) return Q8_OK;  // nothing to compute; empty tensors may carry NULL pointers
-    if (!X || !Wq || !S_w || !Y || !workspace) return Q8_ERR_NULL;
+    if (!X || !Wq || !S_w || !workspace) return Q8_ERR_NULL;
+    if (!Y && !Yq) return Q8_ERR_NULL;
+    if (Yq && !S_y) return Q8_ERR_NULL;
+    if (S_y && !aligned_to(S_y, 4)) return Q8_ERR_ALIGN;
     if (act != Q8_ACT_NONE && act != Q8_ACT_GELU) return Q8_ERR_ARG;
     if (!aligned_to(X, 4) || !aligned_to(Y, 4) || !aligned_to(S_w, 4) || (S_x && !aligned_to(S_x, 4)) ||
         (bias && !aligned_to(bias, 4)) || (dbg_acc && !aligned_to(dbg_acc, 4)) || !aligned_to(workspace, 256))
@@ -97,6 +101,8 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
     g.S_w = S_w;
     g.bias = bias;
     g.Y = Y;
+    g.Yq = Yq;
+    g.S_y = S_y;
     g.dbg_acc = dbg_acc;
     g.status = &hdr->status;
     g.M = M;
@@ -191,15 +197,17 @@ q8_status q8_linear_generic(const float *X, const int8_t *Wq, const float *S_w, 
                        true);
 }
 
-q8_status q8_linear_q(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w, const float *bias,
-                      int act, float *Y, int64_t M, int64_t N, int64_t K, int32_t *dbg_acc, int32_t *dev_status,
-                      void *stream)
+// Body of q8_linear_q / q8_linear_q_requant.
+static q8_status linear_q_impl(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w,
+                               const float *bias, int act, float *Y, int8_t *Yq, const float *S_y, int64_t M, int64_t N,
+                               int64_t K, int32_t *dbg_acc, int32_t *dev_status, void *stream)
 {
     last_launch_info() = LaunchInfo();
     q8_status st = check_gemm_shape(M, N, K);
     if (st != Q8_OK) return st;
     if (M == 0 || N == 0) return Q8_OK;
-    if (!Xq || !S_x || !Wq || !S_w || !Y) return Q8_ERR_NULL;
+    if (!Xq || !S_x || !Wq || !S_w || (!Y && !Yq) || (Yq && !S_y)) return Q8_ERR_NULL;
+    if (S_y && !aligned_to(S_y, 4)) return Q8_ERR_ALIGN;
     if (act != Q8_ACT_NONE && act != Q8_ACT_GELU) return Q8_ERR_ARG;
     if (!aligned_to(Y, 4) || !aligned_to(S_w, 4) || !aligned_to(S_x, 4) || (bias && !aligned_to(bias, 4)) ||
         (dbg_acc && !aligned_to(dbg_acc, 4)) || (dev_status && !aligned_to(dev_status, 4)))
@@ -211,6 +219,8 @@ q8_status q8_linear_q(const int8_t *Xq, const float *S_x, const int8_t *Wq, cons
     g.S_w = S_w;
     g.bias = bias;
     g.Y = Y;
+    g.Yq = Yq;
+    g.S_y = S_y;
     g.dbg_acc = dbg_acc;
     g.status = dev_status;
     g.M = M;
@@ -218,6 +228,31 @@ q8_status q8_linear_q(const int8_t *Xq, const float *S_x, const int8_t *Wq, cons
     g.K = K;
     g.act = act;
     return run_gemm(g, false, static_cast<cudaStream_t>(stream));
+}
+
+q8_status q8_linear_q(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w, const float *bias,
+                      int act, float *Y, int64_t M, int64_t N, int64_t K, int32_t *dbg_acc, int32_t *dev_status,
+                      void *stream)
+{
+    if (M > 0 && N > 0 && !Y) return Q8_ERR_NULL;
+    return linear_q_impl(Xq, S_x, Wq, S_w, bias, act, Y, nullptr, nullptr, M, N, K, dbg_acc, dev_status, stream);
+}
+
+q8_status q8_linear_q_requant(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w,
+                              const float *bias, int act, const float *S_y, int8_t *Yq, float *Y, int64_t M, int64_t N,
+                              int64_t K, int32_t *dbg_acc, int32_t *dev_status, void *stream)
+{
+    if (M > 0 && N > 0 && !Yq) return Q8_ERR_NULL;
+    return linear_q_impl(Xq, S_x, Wq, S_w, bias, act, Y, Yq, S_y, M, N, K, dbg_acc, dev_status, stream);
+}
+
+q8_status q8_linear_requant(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias,
+                            int act, const float *S_y, int8_t *Yq, float *Y, int64_t M, int64_t N, int64_t K,
+                            void *workspace, size_t workspace_bytes, int8_t *dbg_Xq, int32_t *dbg_acc, void *stream)
+{
+    if (M > 0 && N > 0 && !Yq) return Q8_ERR_NULL;
+    return linear_impl(X, Wq, S_w, S_x, bias, act, Y, M, N, K, workspace, workspace_bytes, dbg_Xq, dbg_acc, stream, false,
+                       Yq, S_y);
 }
 
 q8_status q8_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V, int64_t H,
@@ -238,32 +273,63 @@ q8_status q8_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const fl
     return Q8_OK;
 }
 
-q8_status q8_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma, const float *beta,
-                           float eps, int64_t rows, int64_t H, float *out, void *stream)
+static q8_status add_layernorm_impl(const float *x, const float *r1, const float *r2, const float *gamma,
+                                    const float *beta, float eps, int64_t rows, int64_t H, float *out, const float *S_q,
+                                    int8_t *out_q, void *stream)
 {
     last_launch_info() = LaunchInfo();
     if (rows < 0 || H < 0 || H > 12288 || rows > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
     if (rows == 0 || H == 0) return Q8_OK;
-    if (!x || !out) return Q8_ERR_NULL;
+    if (!x || (!out && !out_q) || (out_q && !S_q)) return Q8_ERR_NULL;
     if (!(eps >= 0.0f)) return Q8_ERR_ARG;
     if (!aligned_to(x, 4) || !aligned_to(out, 4) || !aligned_to(r1, 4) || !aligned_to(r2, 4) || !aligned_to(gamma, 4) ||
-        !aligned_to(beta, 4))
+        !aligned_to(beta, 4) || !aligned_to(S_q, 4))
         return Q8_ERR_ALIGN;
-    Q8_CUDA_TRY(launch_add_layernorm(x, r1, r2, gamma, beta, eps, rows, H, out, static_cast<cudaStream_t>(stream)));
+    Q8_CUDA_TRY(launch_add_layernorm(x, r1, r2, gamma, beta, eps, rows, H, out, S_q, out_q,
+                                     static_cast<cudaStream_t>(stream)));
+    last_launch_info().launches = 1;
+    return Q8_OK;
+}
+
+q8_status q8_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma, const float *beta,
+                           float eps, int64_t rows, int64_t H, float *out, void *stream)
+{
+    if (rows > 0 && H > 0 && !out) return Q8_ERR_NULL;
+    return add_layernorm_impl(x, r1, r2, gamma, beta, eps, rows, H, out, nullptr, nullptr, stream);
+}
+
+q8_status q8_add_layernorm_quant(const float *x, const float *r1, const float *r2, const float *gamma,
+                                 const float *beta, float eps, int64_t rows, int64_t H, float *out, const float *S_q,
+                                 int8_t *out_q, void *stream)
+{
+    if (rows > 0 && H > 0 && !out_q) return Q8_ERR_NULL;
+    return add_layernorm_impl(x, r1, r2, gamma, beta, eps, rows, H, out, S_q, out_q, stream);
+}
+
+static q8_status attention_impl(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
+                                int8_t *ctx_q, void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (B < 0 || S < 0 || heads < 0 || B > 65535 || heads > 65535 || S > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
+    if (B == 0 || S == 0 || heads == 0) return Q8_OK;
+    if (!qkv || (!ctx && !ctx_q) || (ctx_q && !S_q)) return Q8_ERR_NULL;
+    if (!aligned_to(qkv, 8) || !aligned_to(ctx, 8) || !aligned_to(S_q, 4)) return Q8_ERR_ALIGN;  // 8-byte vector accesses
+    Q8_CUDA_TRY(launch_attention(qkv, B, S, heads, ctx, S_q, ctx_q, static_cast<cudaStream_t>(stream)));
     last_launch_info().launches = 1;
     return Q8_OK;
 }
 
 q8_status q8_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, void *stream)
 {
-    last_launch_info() = LaunchInfo();
-    if (B < 0 || S < 0 || heads < 0 || B > 65535 || heads > 65535 || S > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
-    if (B == 0 || S == 0 || heads == 0) return Q8_OK;
-    if (!qkv || !ctx) return Q8_ERR_NULL;
-    if (!aligned_to(qkv, 8) || !aligned_to(ctx, 8)) return Q8_ERR_ALIGN;  // 8-byte vector accesses per row of 64
-    Q8_CUDA_TRY(launch_attention(qkv, B, S, heads, ctx, static_cast<cudaStream_t>(stream)));
-    last_launch_info().launches = 1;
-    return Q8_OK;
+    if (B > 0 && S > 0 && heads > 0 && !ctx) return Q8_ERR_NULL;
+    return attention_impl(qkv, B, S, heads, ctx, nullptr, nullptr, stream);
+}
+
+q8_status q8_attention_quant(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
+                             int8_t *ctx_q, void *stream)
+{
+    if (B > 0 && S > 0 && heads > 0 && !ctx_q) return Q8_ERR_NULL;
+    return attention_impl(qkv, B, S, heads, ctx, S_q, ctx_q, stream);
 }
 
 q8_status q8_poll_status(void *dev_status, uint32_t *raw_bits, void *stream)

@@ -91,21 +91,9 @@ __global__ void scale_from_absmax_kernel(const uint32_t *bits, float *S, int32_t
 }
 
 // ------------------------------------------------------------------ Eq. 1
-__device__ __forceinline__ int32_t quantize_one(float x, float S)
-{
-    // one rounded fp32 multiply, nearest-even integer (NaN -> 0, saturating), symmetric clamp
-    int32_t q = __float2int_rn(__fmul_rn(x, S));
-    return max(-127, min(127, q));
-}
+__device__ __forceinline__ int32_t quantize_one(float x, float S) { return quantize_value(x, S); }
 
-__device__ __forceinline__ uint32_t quantize_pack4(float4 v, float S)
-{
-    uint32_t a = (uint32_t)quantize_one(v.x, S) & 0xffu;
-    uint32_t b = (uint32_t)quantize_one(v.y, S) & 0xffu;
-    uint32_t c = (uint32_t)quantize_one(v.z, S) & 0xffu;
-    uint32_t d = (uint32_t)quantize_one(v.w, S) & 0xffu;
-    return a | (b << 8) | (c << 16) | (d << 24);
-}
+__device__ __forceinline__ uint32_t quantize_pack4(float4 v, float S) { return q8::quantize_pack4(v.x, v.y, v.z, v.w, S); }
 
 // VEC: a thread turns one 16-byte load (4 floats) into one 4-byte store, four of them in flight
 // per iteration; consecutive lanes touch consecutive addresses on both sides.

@@ -290,6 +290,8 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
     constexpr int NCHUNK = COLS / 32;
     const int64_t row = row0 + lane;
     const bool row_ok = row < a.M;
+    const float S_y = a.Yq != nullptr ? __ldg(a.S_y) : 1.0f;
+    const bool yq_vec = ((a.N & 15) == 0) && ((reinterpret_cast<uintptr_t>(a.Yq) & 15u) == 0);
 #pragma unroll
     for (int ci = 0; ci < NCHUNK; ++ci) {
         const int64_t nb = col0 + 32 * ci;
@@ -324,6 +326,29 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__fmul_rn(__int2float_rn((int32_t)v[j]), inv));
         }
+        if (a.Yq != nullptr && row_ok) {
+            // re-quantised output for the next quantised layer: Eq. 1 at that layer's activation scale
+            int8_t *qrow = a.Yq + row * a.N + nb;
+            if (yq_vec) {  // N % 16 == 0: a 16-byte piece is never split by the edge
+                if (nb < a.N)
+                    *reinterpret_cast<uint4 *>(qrow) = make_uint4(
+                        quantize_pack4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]), S_y),
+                        quantize_pack4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]), S_y),
+                        quantize_pack4(__uint_as_float(v[8]), __uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]), S_y),
+                        quantize_pack4(__uint_as_float(v[12]), __uint_as_float(v[13]), __uint_as_float(v[14]), __uint_as_float(v[15]), S_y));
+                if (nb + 16 < a.N)
+                    *reinterpret_cast<uint4 *>(qrow + 16) = make_uint4(
+                        quantize_pack4(__uint_as_float(v[16]), __uint_as_float(v[17]), __uint_as_float(v[18]), __uint_as_float(v[19]), S_y),
+                        quantize_pack4(__uint_as_float(v[20]), __uint_as_float(v[21]), __uint_as_float(v[22]), __uint_as_float(v[23]), S_y),
+                        quantize_pack4(__uint_as_float(v[24]), __uint_as_float(v[25]), __uint_as_float(v[26]), __uint_as_float(v[27]), S_y),
+                        quantize_pack4(__uint_as_float(v[28]), __uint_as_float(v[29]), __uint_as_float(v[30]), __uint_as_float(v[31]), S_y));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (nb + j < a.N) qrow[j] = (int8_t)quantize_value(__uint_as_float(v[j]), S_y);
+            }
+        }
+        if (a.Y == nullptr) continue;
         if (tma_store) {
             if (lane == 0) tma_store_wait_read();  // the previous block has left the staging buffer
             __syncwarp();
@@ -666,7 +691,7 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     if (!make_tmap(&tx, a.Xq, a.M, a.K, BLOCK_M) || !make_tmap(&tw, a.Wq, a.N, a.K, C::kBRows))
         return cudaErrorInvalidValue;
     // the TMA store needs a 16-byte aligned base and row pitch; otherwise lanes store their rows directly
-    int tma_store = ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
+    int tma_store = a.Y != nullptr && ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
     if (tma_store) {
         if (!make_tmap_out(&ty, a.Y, a.M, a.N)) return cudaErrorInvalidValue;
     } else {

@@ -32,7 +32,9 @@ struct GemmArgs {
     const float *S_x;   // device scalar
     const float *S_w;   // device scalar
     const float *bias;  // [N] or nullptr
-    float *Y;           // [M,N]
+    float *Y;           // [M,N] fp32 output, or nullptr when only the re-quantised output is wanted
+    int8_t *Yq;         // [M,N] Int8 output Quantize(y | S_y) (Eq. 1 at the consumer's scale), or nullptr
+    const float *S_y;   // device scalar, required with Yq
     int32_t *dbg_acc;   // [M,N] or nullptr
     int32_t *status;    // device status word or nullptr
     int64_t M, N, K;
@@ -61,8 +63,10 @@ cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, co
 
 // ---- fp32 encoder support (q8_support.cu) ----
 cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma,
-                                 const float *beta, float eps, int64_t rows, int64_t H, float *out, cudaStream_t s);
-cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, cudaStream_t s);
+                                 const float *beta, float eps, int64_t rows, int64_t H, float *out, const float *S_q,
+                                 int8_t *out_q, cudaStream_t s);
+cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
+                             int8_t *ctx_q, cudaStream_t s);
 
 // ---- GEMM launchers ----
 bool tcgen05_gemm_supported(const GemmArgs &a);
@@ -73,7 +77,21 @@ cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_
 // The body of q8_linear / q8_linear_generic: validates, quantises X into `workspace`, runs the GEMM (q8_api.cu).
 q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
                       float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
-                      int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic);
+                      int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic, int8_t *Yq = nullptr,
+                      const float *S_y = nullptr);
+
+// Eq. 1 on one value: one rounded fp32 multiply, nearest-even integer (NaN -> 0, saturating), symmetric clamp.
+__device__ __forceinline__ int32_t quantize_value(float x, float S)
+{
+    int32_t q = __float2int_rn(__fmul_rn(x, S));
+    return max(-127, min(127, q));
+}
+
+__device__ __forceinline__ uint32_t quantize_pack4(float a, float b, float c, float d, float S)
+{
+    return ((uint32_t)quantize_value(a, S) & 0xffu) | (((uint32_t)quantize_value(b, S) & 0xffu) << 8) |
+           (((uint32_t)quantize_value(c, S) & 0xffu) << 16) | (((uint32_t)quantize_value(d, S) & 0xffu) << 24);
+}
 
 // ---- epilogue arithmetic shared by both GEMM kernels ----
 // Bias quantised at the product scale: Clamp(nint(b * S_out), -(2^31-1), 2^31-1).

@@ -34,7 +34,8 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_kernel(const float *
                                                                    const float *__restrict__ r2,
                                                                    const float *__restrict__ gamma,
                                                                    const float *__restrict__ beta, float eps, int64_t H,
-                                                                   float *__restrict__ out)
+                                                                   float *__restrict__ out, const float *__restrict__ S_q,
+                                                                   int8_t *__restrict__ out_q)
 {
     extern __shared__ float row[];
     __shared__ float scratch[kLnThreads / 32];
@@ -55,9 +56,13 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_kernel(const float *
     }
     const float var = block_sum(q, scratch) / (float)H;
     const float rstd = 1.0f / sqrtf(var + eps);
+    const float Sq = out_q ? __ldg(S_q) : 1.0f;
     for (int64_t h = threadIdx.x; h < H; h += kLnThreads) {
         const float g = gamma ? gamma[h] : 1.0f, b = beta ? beta[h] : 0.0f;
-        out[base + h] = (row[h] - mean) * rstd * g + b;
+        const float y = (row[h] - mean) * rstd * g + b;
+        if (out) out[base + h] = y;
+        // the same fp32 value, quantised for the next quantised layer (Eq. 1 at that layer's scale)
+        if (out_q) out_q[base + h] = (int8_t)quantize_value(y, Sq);
     }
 }
 
@@ -74,7 +79,8 @@ constexpr int kAttnSmemBytes = (3 * kD * kPitch + kTile * kD) * (int)sizeof(floa
 __device__ __forceinline__ int own_index(int t, int a) { return 2 * t + (a & 1) + 32 * (a >> 1); }
 
 __global__ void __launch_bounds__(256) attention_kernel(const float *__restrict__ qkv, int64_t S, int64_t H,
-                                                        float scale, float *__restrict__ ctx)
+                                                        float scale, float *__restrict__ ctx,
+                                                        const float *__restrict__ S_q, int8_t *__restrict__ ctx_q)
 {
     extern __shared__ __align__(16) float attn_smem[];
     float(*Qt)[kPitch] = reinterpret_cast<float(*)[kPitch]>(attn_smem);                    // Qt[d][i]
@@ -174,29 +180,42 @@ __global__ void __launch_bounds__(256) attention_kernel(const float *__restrict_
         }
     }
 
-    float *obase = ctx + seq * S * H + head * kD;
+    const int64_t obase = seq * S * H + head * kD;
+    const float Sq = ctx_q ? __ldg(S_q) : 1.0f;
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
         const int64_t i = q0 + own_index(ty, a);
         if (i >= S) continue;
         const float inv = 1.0f / l[a];
-        *reinterpret_cast<float2 *>(obase + i * H + 2 * tx) = make_float2(o[a][0] * inv, o[a][1] * inv);
-        *reinterpret_cast<float2 *>(obase + i * H + 2 * tx + 32) = make_float2(o[a][2] * inv, o[a][3] * inv);
+        const float y0 = o[a][0] * inv, y1 = o[a][1] * inv, y2 = o[a][2] * inv, y3 = o[a][3] * inv;
+        const int64_t at = obase + i * H + 2 * tx;
+        if (ctx) {
+            *reinterpret_cast<float2 *>(ctx + at) = make_float2(y0, y1);
+            *reinterpret_cast<float2 *>(ctx + at + 32) = make_float2(y2, y3);
+        }
+        if (ctx_q) {  // the same fp32 values, quantised for the next quantised layer
+            ctx_q[at] = (int8_t)quantize_value(y0, Sq);
+            ctx_q[at + 1] = (int8_t)quantize_value(y1, Sq);
+            ctx_q[at + 32] = (int8_t)quantize_value(y2, Sq);
+            ctx_q[at + 33] = (int8_t)quantize_value(y3, Sq);
+        }
     }
 }
 
 }  // namespace
 
 cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma,
-                                 const float *beta, float eps, int64_t rows, int64_t H, float *out, cudaStream_t s)
+                                 const float *beta, float eps, int64_t rows, int64_t H, float *out, const float *S_q,
+                                 int8_t *out_q, cudaStream_t s)
 {
     if (rows <= 0 || H <= 0) return cudaSuccess;
     add_layernorm_kernel<<<(unsigned)rows, kLnThreads, (size_t)H * sizeof(float), s>>>(x, r1, r2, gamma, beta, eps, H,
-                                                                                       out);
+                                                                                       out, S_q, out_q);
     return cudaGetLastError();
 }
 
-cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, cudaStream_t s)
+cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
+                             int8_t *ctx_q, cudaStream_t s)
 {
     if (B <= 0 || S <= 0 || heads <= 0) return cudaSuccess;
     static bool attr_set[64] = {};  // opt-in shared-memory size: per device, per function
@@ -210,7 +229,7 @@ cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t hea
         attr_set[dev] = true;
     }
     dim3 grid((unsigned)((S + kTile - 1) / kTile), (unsigned)heads, (unsigned)B);
-    attention_kernel<<<grid, 256, kAttnSmemBytes, s>>>(qkv, S, heads * kD, 1.0f / 8.0f, ctx);
+    attention_kernel<<<grid, 256, kAttnSmemBytes, s>>>(qkv, S, heads * kD, 1.0f / 8.0f, ctx, S_q, ctx_q);
     return cudaGetLastError();
 }
 

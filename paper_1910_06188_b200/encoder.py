@@ -122,7 +122,46 @@ class Q8BertEncoder:
             q8.q8_add_layernorm(bf["f2"], bf["h1"], eps=LN_EPS, out=bf["h"])
         return bf["h"]
 
-    def launches_per_forward(self, scales: str = "static") -> int:
+    def forward_fused(self, ids: torch.Tensor, B: int, S: int) -> torch.Tensor:
+        """The same forward with static (Eq. 4) scales and every quantiser folded into the kernel that produces
+        its input: LayerNorm and attention also emit Int8 at the consuming FC's scale, FFN1 emits only Int8 at
+        FFN2's scale.  No stand-alone quantise pass is left and FFN1's fp32 output never reaches HBM.  The
+        Int8 tensors are identical to those of forward(), so the result is bit-identical too."""
+        T = B * S
+        bf = self._buffers(T)
+        if "hq" not in bf:
+            i8 = lambda n: torch.empty((T, n), dtype=torch.int8, device=self.device)
+            bf.update(hq=i8(self.H), ctxq=i8(self.H), h1q=i8(self.H), fq=i8(self.F))
+        sx = lambda l, name: q8.calibrate_S_x(self.layers[l][name]["state"])
+        pos_ids = torch.arange(S, dtype=torch.int32, device=self.device).repeat(B)
+        typ_ids = torch.zeros(T, dtype=torch.int32, device=self.device)
+        q8.q8_embedding(ids, self.word, self.S_word, out=bf["ew"], dev_status=bf["status"])
+        q8.q8_embedding(pos_ids, self.pos, self.S_pos, out=bf["ep"], dev_status=bf["status"])
+        q8.q8_embedding(typ_ids, self.typ, self.S_typ, out=bf["et"], dev_status=bf["status"])
+        q8.q8_add_layernorm_quant(bf["ew"], bf["ep"], bf["et"], sx(0, "qkv"), out_q=bf["hq"], out=bf["h"], eps=LN_EPS)
+        st = bf["status"]
+        for l in range(self.L):
+            p = self.layers[l]
+            q8.q8_linear_q(bf["hq"], sx(l, "qkv"), p["qkv"]["Wq"], p["qkv"]["S_w"], p["qkv"]["b"], 0, Y=bf["qkv"],
+                           dev_status=st)
+            q8.q8_attention_quant(bf["qkv"], B, S, self.heads, sx(l, "attn_out"), ctx_q=bf["ctxq"])
+            q8.q8_linear_q(bf["ctxq"], sx(l, "attn_out"), p["attn_out"]["Wq"], p["attn_out"]["S_w"], p["attn_out"]["b"],
+                           0, Y=bf["ao"], dev_status=st)
+            q8.q8_add_layernorm_quant(bf["ao"], bf["h"], None, sx(l, "ffn1"), out_q=bf["h1q"], out=bf["h1"], eps=LN_EPS)
+            q8.q8_linear_q_requant(bf["h1q"], sx(l, "ffn1"), p["ffn1"]["Wq"], p["ffn1"]["S_w"], p["ffn1"]["b"], 1,
+                                   sx(l, "ffn2"), Yq=bf["fq"], dev_status=st)
+            q8.q8_linear_q(bf["fq"], sx(l, "ffn2"), p["ffn2"]["Wq"], p["ffn2"]["S_w"], p["ffn2"]["b"], 0, Y=bf["f2"],
+                           dev_status=st)
+            if l + 1 < self.L:
+                q8.q8_add_layernorm_quant(bf["f2"], bf["h1"], None, sx(l + 1, "qkv"), out_q=bf["hq"], out=bf["h"],
+                                          eps=LN_EPS)
+            else:
+                q8.q8_add_layernorm(bf["f2"], bf["h1"], eps=LN_EPS, out=bf["h"])
+        return bf["h"]
+
+    def launches_per_forward(self, scales: str = "static", fused: bool = False) -> int:
+        if fused:
+            return 4 + self.L * 7
         per_fc = 2 if scales == "static" else (4 if scales == "dynamic" else 6)
         return 4 + self.L * (4 * per_fc + 3)
 

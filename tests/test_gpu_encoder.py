@@ -164,3 +164,58 @@ def test_bert_base_encoder_forward():
 def test_bert_large_encoder_forward():
     """BERT-Large encoder, batch 64 x seq 384, EMA scales (decay 0.9999) over 16 seeded batches."""
     _run_model_case(synth.BERT_LARGE, config=5, B=64, S=384, scales="static", calib_batches=16)
+
+
+# ------------------------------------------------------------------ fused re-quantisation
+def test_requantising_outputs_equal_quantising_the_fp32_output():
+    """Each producer's Int8 output must be Eq. 1 applied to exactly the fp32 value it would have stored."""
+    S_q = dev(np.array([9.5], np.float32))
+    # LayerNorm
+    x, r1 = synth.activation(300, 768, 4000), synth.activation(300, 768, 4001)
+    out = torch.empty((300, 768), device="cuda")
+    oq = q8.q8_add_layernorm_quant(dev(x), dev(r1), None, S_q, out=out)
+    assert_close_fp(out.cpu().numpy(), o.add_layernorm(x, r1), "LN fp32")
+    assert np.array_equal(oq.cpu().numpy(), o.quantize(out.cpu().numpy(), 9.5))
+    assert torch.equal(q8.q8_add_layernorm_quant(dev(x), dev(r1), None, S_q), oq)          # Int8 only
+    # attention
+    B, S, heads = 2, 70, 3
+    qkv = synth.normal((B * S, 3 * heads * 64), 1.0, 4010)
+    ctx = torch.empty((B * S, heads * 64), device="cuda")
+    cq = q8.q8_attention_quant(dev(qkv), B, S, heads, S_q, ctx=ctx)
+    assert_close_fp(ctx.cpu().numpy(), o.attention(qkv, B, S, heads), "attention fp32")
+    assert np.array_equal(cq.cpu().numpy(), o.quantize(ctx.cpu().numpy(), 9.5))
+    assert torch.equal(q8.q8_attention_quant(dev(qkv), B, S, heads, S_q), cq)
+    # quantised FC, fp32 in and Int8 in, with and without GELU, tensor-core and generic kernels
+    for (M, N, K, act) in [(515, 1040, 272, 1), (300, 208, 400, 0), (64, 50, 33, 1)]:
+        X, W, b = synth.activation(M, K, 4020 + M), synth.weight(N, K, 4021 + M), synth.bias(N, 4022 + M)
+        Wq_ref, S_w_ref, _ = o.quantize_weight(W)
+        S_x = np.float32(20.0)
+        ref = o.linear(X, Wq_ref, S_w_ref, S_x, b, act)
+        Wq, S_w = q8.q8_quantize_weight(dev(W))
+        Sx_d = dev(np.array([S_x], np.float32))
+        S_y = dev(np.array([31.0], np.float32))
+        Y = torch.empty((M, N), device="cuda")
+        Yq = q8.q8_linear_requant(dev(X), Wq, S_w, Sx_d, dev(b), act, S_y, Y=Y)
+        assert_close_fp(Y.cpu().numpy(), ref["y"], "requant fp32 copy")
+        want_q = o.quantize(Y.cpu().numpy(), 31.0)
+        assert np.array_equal(Yq.cpu().numpy(), want_q)
+        assert torch.equal(q8.q8_linear_requant(dev(X), Wq, S_w, Sx_d, dev(b), act, S_y), Yq)   # Int8 only
+        Xq, _ = q8.q8_quantize_activation(dev(X), Sx_d)
+        assert torch.equal(q8.q8_linear_q_requant(Xq, Sx_d, Wq, S_w, dev(b), act, S_y), Yq)
+        # against the oracle's own fp64 output the Int8 values may differ by one step only where y * S_y
+        # sits within fp32 rounding of a tie
+        exact = o.quantize(ref["y"].astype(np.float32), 31.0).astype(np.int32)
+        d = np.abs(exact - Yq.cpu().numpy().astype(np.int32))
+        assert d.max() <= 1 and (d != 0).mean() < 1e-3
+
+
+def test_fused_forward_is_bit_identical_to_the_unfused_one():
+    dims = dict(hidden=128, ffn=512, heads=2, layers=3, vocab=500, max_pos=96)
+    for dims_, cfg, B, S in [(dims, 31, 3, 70), (synth.BERT_BASE, 3, 32, 128)]:
+        enc = enc_mod.Q8BertEncoder(dims_, config=cfg)
+        ids = enc_mod.random_ids(B * S, dims_["vocab"], cfg)
+        enc.forward(ids, B, S, scales="calibrate")
+        want = enc.forward(ids, B, S, scales="static").clone()
+        got = enc.forward_fused(ids, B, S)
+        assert enc.poll() == ((q8.Q8_OK, 0), (q8.Q8_OK, 0))
+        assert torch.equal(got, want)
