@@ -453,6 +453,18 @@ def measure_encoders(args, torch, q8):
         e1.record()
         torch.cuda.synchronize()
         ms_fused = e0.elapsed_time(e1) / reps
+        # ... and replayed from a CUDA graph (removes the host launch cost, which dominates the small model)
+        graph, _ = enc.capture(ids, B, S)
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms_graph = e0.elapsed_time(e1) / reps
+        del graph
         codes = enc.poll()
         # breakdown: time the three kinds of calls of one forward
         shares = {"q8_linear": 0.0, "attention_fp32": 0.0, "layernorm_embedding": 0.0}
@@ -484,6 +496,7 @@ def measure_encoders(args, torch, q8):
         out[name] = {
             "tokens_per_s": T / (ms * 1e-3), "ms_per_forward": ms, "layers": enc.L, "tokens": T,
             "tokens_per_s_fused_requant": T / (ms_fused * 1e-3), "ms_per_forward_fused_requant": ms_fused,
+            "tokens_per_s_fused_cuda_graph": T / (ms_graph * 1e-3), "ms_per_forward_fused_cuda_graph": ms_graph,
             "gpu_launches_per_forward": enc.launches_per_forward(),
             "gpu_launches_per_forward_fused_requant": enc.launches_per_forward(fused=True),
             "status": [list(c) for c in codes],

@@ -159,6 +159,18 @@ class Q8BertEncoder:
                 q8.q8_add_layernorm(bf["f2"], bf["h1"], eps=LN_EPS, out=bf["h"])
         return bf["h"]
 
+    def capture(self, ids: torch.Tensor, B: int, S: int, fused: bool = True):
+        """Captures one static-scale forward into a CUDA graph (the forward is a fixed sequence of launches on
+        fixed buffers, and for small batches the host cannot issue them as fast as the GPU runs them).
+        Returns (graph, output tensor); graph.replay() recomputes the output from the current contents of `ids`."""
+        run = (lambda: self.forward_fused(ids, B, S)) if fused else (lambda: self.forward(ids, B, S))
+        run()                                   # first-call set-up (function attributes, buffers) outside capture
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            out = run()
+        return graph, out
+
     def launches_per_forward(self, scales: str = "static", fused: bool = False) -> int:
         if fused:
             return 4 + self.L * 7

@@ -219,3 +219,13 @@ def test_fused_forward_is_bit_identical_to_the_unfused_one():
         got = enc.forward_fused(ids, B, S)
         assert enc.poll() == ((q8.Q8_OK, 0), (q8.Q8_OK, 0))
         assert torch.equal(got, want)
+        # and replayed from a CUDA graph, also after the token ids change in place
+        graph, out = enc.capture(ids, B, S)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, want)
+        ids.copy_(torch.flip(ids, dims=[0]))
+        graph.replay()
+        torch.cuda.synchronize()
+        replayed = out.clone()
+        assert torch.equal(replayed, enc.forward(ids, B, S, scales="static"))
