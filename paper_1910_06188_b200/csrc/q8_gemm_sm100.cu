@@ -32,13 +32,17 @@ constexpr int BLOCK_M = 128;       // accumulator rows per CTA: row i <-> TMEM l
 constexpr int BLOCK_K = 128;       // bytes == int8 elements per stage row: one 128-byte swizzle span
 constexpr int UMMA_K = 32;         // K of one kind::i8 instruction
 constexpr int kAccStages = 2;      // TMEM accumulator double buffering
-constexpr int kEpilogueWarps = 8;  // two per TMEM lane quarter, each taking half of the tile's columns
-constexpr int kThreads = 64 + 32 * kEpilogueWarps;
+// Epilogue warps per CTA (template parameter EW): 8 = two per TMEM lane quarter, each taking half of the tile's
+// columns; 16 = four per quarter.  A warp walks its 32-column blocks one after the other and every block is a
+// chain of dependent latencies (TMEM load, arithmetic, staging, proxy fence, TMA store), so when the main loop is
+// short (small K) more warps shorten the epilogue; the extra staging buffers cost one stage of the operand ring.
 constexpr int kStagingBytesPerWarp = 32 * 32 * 4;  // the 32 x 32 fp32 block one tcgen05.ld hands to a warp
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
-template <int BLOCK_N, int CTAS>
+template <int BLOCK_N, int CTAS, int EW>
 struct Cfg {
+    static constexpr int kEpilogueWarps = EW;
+    static constexpr int kThreads = 64 + 32 * EW;
     static constexpr int kBRows = BLOCK_N / CTAS;  // W_q rows each CTA loads
     static constexpr int kABytes = BLOCK_M * BLOCK_K;
     static constexpr int kBBytes = kBRows * BLOCK_K;
@@ -51,7 +55,7 @@ struct Cfg {
     static constexpr int kBarrierBytes = (2 * kStages + 2 * kAccStages) * 8 + 16;
     // +1024: the dynamic shared window is only 16-byte aligned; tiles need 1024 (swizzle atom)
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kStagingBytes + kBiasBytes + kBarrierBytes;
-    static constexpr int kColsPerWarp = BLOCK_N / 2 < 32 ? 32 : BLOCK_N / 2;  // BLOCK_N = 32 leaves half the warps idle
+    static constexpr int kColsPerWarp = BLOCK_N / (EW / 4) < 32 ? 32 : BLOCK_N / (EW / 4);  // narrow tiles idle some warps
     static_assert((kTmemCols & (kTmemCols - 1)) == 0 && kTmemCols <= 512, "TMEM columns: power of two <= 512");
     static_assert(BLOCK_N % 32 == 0 && BLOCK_N >= 32 && BLOCK_N <= 256, "UMMA N");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -370,12 +374,13 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int BLOCK_N, int CTAS>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int BLOCK_N, int CTAS, int EW>
+__global__ void __launch_bounds__(64 + 32 * EW, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ CUtensorMap tmap_y, GemmArgs a, int tma_store)
 {
-    using C = Cfg<BLOCK_N, CTAS>;
+    using C = Cfg<BLOCK_N, CTAS, EW>;
+    constexpr int kEpilogueWarps = EW;
     constexpr int TILE_M = BLOCK_M * CTAS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -650,12 +655,14 @@ int sm_count()
 }
 
 int g_force_block_n = 0, g_force_ctas = 0;  // set by q8_tune_gemm_tile(); 0 = choose automatically
+int g_force_epilogue_warps = 0;            // 0 automatic, else 8 or 16 (cta_group::2 kernel only)
 
-template <int BLOCK_N, int CTAS>
+template <int BLOCK_N, int CTAS, int EW = 8>
 cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
 {
-    using C = Cfg<BLOCK_N, CTAS>;
-    auto kernel = gemm_tcgen05_kernel<BLOCK_N, CTAS>;
+    using C = Cfg<BLOCK_N, CTAS, EW>;
+    constexpr int kThreads = C::kThreads;
+    auto kernel = gemm_tcgen05_kernel<BLOCK_N, CTAS, EW>;
     static bool attr_set[64] = {};  // the opt-in shared-memory size is a per-device, per-function attribute
     static int max_units[64] = {};  // co-resident CTAs (CTAS = 1) or CTA pairs (CTAS = 2) on the device
     int dev = 0;
@@ -716,6 +723,7 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     li.gemm_kernel = 1;
     li.block_n = BLOCK_N;
     li.ctas = CTAS;
+    li.epilogue_warps = EW;
     li.grid = units * CTAS;
     li.launches += 1;
     return e;
@@ -731,7 +739,11 @@ double tile_step_cost(int bn)
 
 cudaError_t launch_by_shape(int bn, int ctas, const GemmArgs &a, cudaStream_t s)
 {
-    if (ctas == 2) return launch_cfg<256, 2>(a, s);
+    if (ctas == 2) {
+        // a short main loop (small K) leaves the epilogue on the critical path: give it twice the warps
+        const bool wide_epilogue = g_force_epilogue_warps ? g_force_epilogue_warps == 16 : a.K <= 2048;
+        return wide_epilogue ? launch_cfg<256, 2, 16>(a, s) : launch_cfg<256, 2, 8>(a, s);
+    }
     switch (bn) {
         case 256: return launch_cfg<256, 1>(a, s);
         case 128: return launch_cfg<128, 1>(a, s);
@@ -742,10 +754,11 @@ cudaError_t launch_by_shape(int bn, int ctas, const GemmArgs &a, cudaStream_t s)
 
 }  // namespace
 
-void set_gemm_tile_override(int block_n, int ctas)
+void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps)
 {
     g_force_block_n = block_n;
     g_force_ctas = ctas;
+    g_force_epilogue_warps = epilogue_warps;
 }
 
 bool tcgen05_gemm_supported(const GemmArgs &a)

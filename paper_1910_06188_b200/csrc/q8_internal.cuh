@@ -46,6 +46,7 @@ struct LaunchInfo {
     int launches = 0;
     int block_n = 0;
     int ctas = 0;  // CTAs cooperating on one tile (1, or 2 for cta_group::2)
+    int epilogue_warps = 0;
     int grid = 0;
 };
 LaunchInfo &last_launch_info();
@@ -70,7 +71,7 @@ cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t hea
 
 // ---- GEMM launchers ----
 bool tcgen05_gemm_supported(const GemmArgs &a);
-void set_gemm_tile_override(int block_n, int ctas);  // 0, 0 = automatic choice
+void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps = 0);  // 0, 0 = automatic choice
 cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s);  // q8_gemm_sm100.cu
 cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_generic.cu
 
