@@ -223,14 +223,37 @@ def run_ours(args):
 
     launches_per_step = 0
 
+    # The four FC layers of the set (and the embedding gather) are independent of one another, so with
+    # --streams > 1 each runs on its own stream: the HBM-bound quantise / gather passes of one layer overlap the
+    # GEMM of another.  Every step forks from and joins back into the timed stream.
+    side = [torch.cuda.Stream(device=dev) for _ in range(max(0, min(args.streams, 5) - 1))]
+    fork, joins = torch.cuda.Event(), [torch.cuda.Event() for _ in side]
+
     def step():
         nonlocal launches_per_step
         n = 0
-        q8.q8_embedding(ids, Eq, S_e, out=emb_out)
-        n += q8.q8_last_launch_info()["launches"]
+        work = [lambda: q8.q8_embedding(ids, Eq, S_e, out=emb_out)]
         for L in layers:
-            q8.q8_linear(L["Xd"], L["Wq"], L["S_w"], L["S_x"], L["bd"], L["act"], Y=L["Y"], workspace=L["ws"])
-            n += q8.q8_last_launch_info()["launches"]
+            work.append(lambda L=L: q8.q8_linear(L["Xd"], L["Wq"], L["S_w"], L["S_x"], L["bd"], L["act"], Y=L["Y"],
+                                                 workspace=L["ws"]))
+        if not side:
+            for w in work:
+                w()
+                n += q8.q8_last_launch_info()["launches"]
+        else:
+            # biggest jobs first (FFN2's 503 MB quantise pass, then FFN1), round-robin over main + side streams
+            order = sorted(range(len(work)), key=lambda i: -(layers[i - 1]["M"] * layers[i - 1]["K"] if i else 0))
+            fork.record(stream)
+            lanes = [stream] + side
+            for s_ in side:
+                s_.wait_event(fork)
+            for j, i in enumerate(order):
+                with torch.cuda.stream(lanes[j % len(lanes)]):
+                    work[i]()
+                    n += q8.q8_last_launch_info()["launches"]
+            for s_, ev in zip(side, joins):
+                ev.record(s_)
+                stream.wait_event(ev)
         launches_per_step = n
 
     def barrier():
@@ -388,13 +411,14 @@ def run_ours(args):
         }
 
     # ---- whole encoder forwards (tokens/s): int8 embeddings, every FC quantised, attention / LayerNorm in fp32
-    encoder = None
+    encoder = small = None
     if world == 1 and not args.no_encoder:
         for L in layers:
             L.clear()
         del host_in, host_out, host_emb, emb_out
         torch.cuda.empty_cache()
         encoder = measure_encoders(args, torch, q8)
+        small = measure_small_cases(args, torch, q8)
 
     line = {
         "metric": "q8_linear_int8_tops", "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
@@ -405,6 +429,7 @@ def run_ours(args):
             "tokens_per_s": M * world / (ms_per_step * 1e-3),
             "l2": "inputs larger than L2 (each step reads ~0.9 GB and writes ~1.0 GB; L2 is 126 MB)",
             "step": "q8_embedding + 4 x q8_linear (quantise, tcgen05 GEMM, fused epilogue), static scales",
+            "streams": max(1, min(args.streams, 5)),
         },
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -413,11 +438,71 @@ def run_ours(args):
         "roofline": roofline,
         "cpu_baseline": cpu_baseline,
         "encoder": encoder,
+        "small_cases": small,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
     return 0
+
+
+def measure_small_cases(args, torch, q8):
+    """The two smaller BASELINE configurations, timed as back-to-back calls (their data fits in L2, so these are
+    L2-warm, launch-latency-dominated figures; reported in microseconds rather than against a roofline)."""
+    out = {}
+    dev = torch.device("cuda", torch.cuda.current_device())
+
+    def timed(fn, reps):
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e3
+
+    # config 1: one layer, X [128 x 768], dynamic scale (Sec. 4.1): absmax, scale, quantise, GEMM
+    X = torch.from_numpy(synth.activation(128, 768, synth.seed_for(1, 0))).to(dev)
+    Wq, S_w = q8.q8_quantize_weight(torch.from_numpy(synth.weight(768, 768, synth.seed_for(1, 1))).to(dev))
+    b = torch.from_numpy(synth.bias(768, synth.seed_for(1, 2))).to(dev)
+    Y = torch.empty((128, 768), device=dev)
+    ws = q8.new_workspace(128, 768, 768, dev)
+    us = timed(lambda: q8.q8_linear(X, Wq, S_w, None, b, 0, Y=Y, workspace=ws), 200)
+    info = q8.q8_last_launch_info()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        q8.q8_linear(X, Wq, S_w, None, b, 0, Y=Y, workspace=ws)
+    us_graph = timed(graph.replay, 200)
+    out["single_layer_128x768x768_dynamic"] = {"us_per_call": us, "us_per_call_cuda_graph": us_graph,
+                                               "launches": info["launches"], "block_n": info["block_n"],
+                                               "grid": info["grid"], "tops": 2.0 * 128 * 768 * 768 / us_graph / 1e6}
+    del graph
+    # config 2: BERT-Base FC set, M = 4096, static scales
+    M, layers = make_layers(2, synth.BERT_BASE)
+    for L in layers:
+        L["Xd"] = torch.from_numpy(L["X"]).to(dev)
+        L["bd"] = torch.from_numpy(L["b"]).to(dev)
+        L["Wq"], L["S_w"] = q8.q8_quantize_weight(torch.from_numpy(L["W"]).to(dev))
+        st = q8.new_calibrate_state(dev)
+        q8.q8_calibrate(torch.from_numpy(L["calib"]).to(dev), 0.9999, st)
+        L["S_x"] = q8.calibrate_S_x(st).clone()
+        L["Y"] = torch.empty((M, L["N"]), device=dev)
+        L["ws"] = q8.new_workspace(M, L["N"], L["K"], dev)
+
+    def step():
+        for L in layers:
+            q8.q8_linear(L["Xd"], L["Wq"], L["S_w"], L["S_x"], L["bd"], L["act"], Y=L["Y"], workspace=L["ws"])
+    us = timed(step, 100)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    us_graph = timed(graph.replay, 100)
+    out["bert_base_fc_set_m4096"] = {"us_per_step": us, "us_per_step_cuda_graph": us_graph,
+                                     "tops": total_ops(layers) / us_graph / 1e6, "note": "L2-warm"}
+    return out
 
 
 def measure_encoders(args, torch, q8):
@@ -521,6 +606,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-encoder", action="store_true", help="skip the whole-encoder tokens/s measurement")
     ap.add_argument("--encoder-steps", type=int, default=5)
+    ap.add_argument("--streams", type=int, default=1,
+                    help="streams used inside a step for the independent layers of the FC set (1 = serial)")
     ap.add_argument("--layers", default="", help="comma list of FC layers to keep (qkv,attn_out,ffn1,ffn2); default all")
     ap.add_argument("--profile-mode", action="store_true",
                     help="only warm-up + timed steps (no per-kernel pass, e2e or CPU baseline): for ncu captures")
