@@ -80,6 +80,15 @@ q8_status q8_quantize_activation(const float *X, int64_t numel, const float *S_x
 q8_status q8_calibrate(const float *X, int64_t numel, float decay, void *state, void *stream);
 size_t q8_calibrate_state_bytes(void);
 
+/* Training-mode building blocks (Sec. 2.2 and the training sentence of Sec. 3).
+ * q8_fake_quantize: Xhat = Quantize(X | S) / S, the rounding of Eq. 1 simulated in fp32 (X, Xhat flat fp32 of
+ *   `numel` elements, may alias; S a device scalar, e.g. &state->S_x kept current by q8_calibrate, which is the
+ *   EMA update of Eq. 4 that training performs on every forward).
+ * q8_ste_backward: the straight-through estimator of Eq. 5, d Xhat / d X = 1: grad_in = grad_out (a device copy;
+ *   a no-op when the two pointers are equal). */
+q8_status q8_fake_quantize(const float *X, int64_t numel, const float *S, float *Xhat, void *stream);
+q8_status q8_ste_backward(const float *grad_out, int64_t numel, float *grad_in, void *stream);
+
 /* The quantised fully-connected layer in inference mode (Sec. 3):
  *   X_q = Quantize(X | S_x)  (Eq. 1);  acc = X_q W_q^T in Int32, accumulated onto the Int32 bias
  *   b_q = Clamp(nint(b * fl32(S_x * S_w)), -(2^31-1), 2^31-1);  Y = (acc + b_q) / (S_x * S_w);
@@ -160,6 +169,21 @@ q8_status q8_add_layernorm(const float *x, const float *r1, const float *r2, con
  *   qkv [B*S, 3*H] = [q | k | v] per token (H = heads * 64), ctx [B*S, H] (written):
  *   ctx[b, i, h*64 : h*64+64] = sum_j softmax_j(q_i . k_j / 8) v_j  over the S tokens of sequence b. */
 q8_status q8_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, void *stream);
+
+/* Weight scales per block of output rows.  Eq. 3 gives every FC layer of the paper its own S_w; when several
+ * layers that share an input are stored as one matrix (the fused QKV projection: three layers of H rows each),
+ * one scale per block of `seg_rows` rows keeps exactly the paper's per-layer scales: the result equals running
+ * the blocks as separate quantised FC layers.  S_w is then an array of ceil(N / seg_rows) device floats.
+ * The tensor-core kernel needs seg_rows % 32 == 0; other values run the generic kernel. */
+q8_status q8_quantize_weight_segments(const float *W, int64_t N, int64_t K, int64_t seg_rows, int8_t *Wq,
+                                      float *S_w, int32_t *dev_status, void *stream);
+q8_status q8_linear_wseg(const float *X, const int8_t *Wq, const float *S_w, int64_t w_seg_rows,
+                         const float *S_x, const float *bias, int act, float *Y, int64_t M, int64_t N,
+                         int64_t K, void *workspace, size_t workspace_bytes, int8_t *dbg_Xq, int32_t *dbg_acc,
+                         void *stream);
+q8_status q8_linear_q_wseg(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w,
+                           int64_t w_seg_rows, const float *bias, int act, float *Y, int64_t M, int64_t N,
+                           int64_t K, int32_t *dbg_acc, int32_t *dev_status, void *stream);
 
 /* Fused re-quantisation (Sec. 3 inference mode chained layer to layer; Eq. 1 with the consumer's Eq. 4
  * scale): the producer of an activation also emits it as Int8 at the NEXT quantised layer's static

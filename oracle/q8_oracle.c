@@ -288,3 +288,17 @@ void q8o_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, int64_
         }
     }
 }
+
+/* ---- Training-mode pieces (Sec. 2.2, Sec. 3 "During training ..."): fake quantisation simulates the rounding
+ * in floating point, x_hat = Quantize(x | S, M) / S, and the straight-through estimator (Eq. 5) passes the
+ * gradient through unchanged. ---- */
+void q8o_fake_quantize(const float *x, int64_t n, float S, double *xhat)
+{
+    for (int64_t i = 0; i < n; ++i) xhat[i] = (double)q8o_quantize_one(x[i], S) / (double)S;
+}
+
+/* Eq. 5: d x_hat / d x = 1 for every element. */
+void q8o_ste_backward(const float *grad_out, int64_t n, double *grad_in)
+{
+    for (int64_t i = 0; i < n; ++i) grad_in[i] = (double)grad_out[i];
+}

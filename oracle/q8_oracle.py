@@ -67,6 +67,10 @@ def lib() -> C.CDLL:
         L.q8o_add_layernorm.argtypes = [fp, fp, fp, fp, fp, C.c_double, C.c_int64, C.c_int64, dp]
         L.q8o_attention.restype = None
         L.q8o_attention.argtypes = [fp, C.c_int64, C.c_int64, C.c_int64, C.c_int64, dp]
+        L.q8o_fake_quantize.restype = None
+        L.q8o_fake_quantize.argtypes = [fp, C.c_int64, C.c_float, dp]
+        L.q8o_ste_backward.restype = None
+        L.q8o_ste_backward.argtypes = [fp, C.c_int64, dp]
         _lib = L
     return _lib
 
@@ -233,3 +237,18 @@ def attention(qkv, B: int, S: int, heads: int, d: int = 64) -> np.ndarray:
     ctx = np.empty((B * S, heads * d), np.float64)
     lib().q8o_attention(_p(qkv, C.c_float), B, S, heads, d, _p(ctx, C.c_double))
     return ctx
+
+
+def fake_quantize(x, S) -> np.ndarray:
+    """Training-mode fake quantisation x_hat = Quantize(x | S) / S (fp64)."""
+    x = _f32(x)
+    out = np.empty(x.shape, np.float64)
+    lib().q8o_fake_quantize(_p(x, C.c_float), x.size, C.c_float(float(np.float32(S))), _p(out, C.c_double))
+    return out
+
+
+def ste_backward(grad_out) -> np.ndarray:
+    g = _f32(grad_out)
+    out = np.empty(g.shape, np.float64)
+    lib().q8o_ste_backward(_p(g, C.c_float), g.size, _p(out, C.c_double))
+    return out

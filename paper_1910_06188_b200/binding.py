@@ -26,6 +26,8 @@ _vp, _i64, _sz, _int, _f = C.c_void_p, C.c_int64, C.c_size_t, C.c_int, C.c_float
 SIGNATURES = {
     "q8_quantize_weight": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp]),
     "q8_quantize_activation": (_int, [_vp, _i64, _vp, _vp, _vp, _vp, _vp]),
+    "q8_fake_quantize": (_int, [_vp, _i64, _vp, _vp, _vp]),
+    "q8_ste_backward": (_int, [_vp, _i64, _vp, _vp]),
     "q8_calibrate": (_int, [_vp, _i64, _f, _vp, _vp]),
     "q8_calibrate_state_bytes": (_sz, []),
     "q8_linear": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
@@ -36,6 +38,9 @@ SIGNATURES = {
     "q8_embedding": (_int, [_vp, _i64, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _vp]),
     "q8_add_layernorm": (_int, [_vp, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp]),
     "q8_attention": (_int, [_vp, _i64, _i64, _i64, _vp, _vp]),
+    "q8_quantize_weight_segments": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "q8_linear_wseg": (_int, [_vp, _vp, _vp, _i64, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
+    "q8_linear_q_wseg": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _int, _vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "q8_linear_requant": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
     "q8_linear_q_requant": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "q8_add_layernorm_quant": (_int, [_vp, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp, _vp, _vp]),
@@ -139,6 +144,26 @@ def q8_quantize_activation(X: torch.Tensor, S_x: Optional[torch.Tensor] = None, 
                                        _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "q8_quantize_activation")
     return Xq, (S_x_used if S_x_used is not None else S_x)
+
+
+def q8_fake_quantize(X, S, Xhat=None, stream=None):
+    """Training-mode fake quantisation: Xhat = Quantize(X | S) / S."""
+    if Xhat is None:
+        Xhat = torch.empty_like(X)
+    st = load().q8_fake_quantize(_ptr(X, torch.float32, "X"), X.numel(), _ptr(S, torch.float32, "S"),
+                                 _ptr(Xhat, torch.float32, "Xhat"), _stream(stream))
+    _check(st, "q8_fake_quantize")
+    return Xhat
+
+
+def q8_ste_backward(grad_out, grad_in=None, stream=None):
+    """Straight-through estimator (Eq. 5): the gradient of fake quantisation is the incoming gradient."""
+    if grad_in is None:
+        grad_in = torch.empty_like(grad_out)
+    st = load().q8_ste_backward(_ptr(grad_out, torch.float32, "grad_out"), grad_out.numel(),
+                                _ptr(grad_in, torch.float32, "grad_in"), _stream(stream))
+    _check(st, "q8_ste_backward")
+    return grad_in
 
 
 def q8_calibrate_state_bytes() -> int:
@@ -283,6 +308,50 @@ def q8_attention(qkv, B: int, S: int, heads: int, ctx=None, stream=None):
                              _stream(stream))
     _check(st, "q8_attention")
     return ctx
+
+
+def q8_quantize_weight_segments(W, seg_rows: int, dev_status=None, stream=None):
+    """Eq. 3 + Eq. 1 with one scale per block of `seg_rows` output rows; returns (W_q, S_w[ceil(N/seg_rows)])."""
+    N, K = W.shape
+    Wq = torch.empty((N, K), dtype=torch.int8, device=W.device)
+    S_w = torch.empty((N + seg_rows - 1) // seg_rows, dtype=torch.float32, device=W.device)
+    st = load().q8_quantize_weight_segments(_ptr(W, torch.float32, "W"), N, K, int(seg_rows), _ptr(Wq, torch.int8, "Wq"),
+                                            _ptr(S_w, torch.float32, "S_w"), _ptr(dev_status, torch.int32, "dev_status"),
+                                            _stream(stream))
+    _check(st, "q8_quantize_weight_segments")
+    return Wq, S_w
+
+
+def q8_linear_wseg(X, Wq, S_w, seg_rows: int, S_x=None, bias=None, act: int = Q8_ACT_NONE, Y=None, workspace=None,
+                   dbg_Xq=None, dbg_acc=None, stream=None):
+    """q8_linear with one weight scale per block of `seg_rows` output features."""
+    M, K = X.shape
+    N = Wq.shape[0]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float32, device=X.device)
+    if workspace is None:
+        workspace = new_workspace(M, N, K, X.device)
+    st = load().q8_linear_wseg(_ptr(X, torch.float32, "X"), _ptr(Wq, torch.int8, "Wq"), _ptr(S_w, torch.float32, "S_w"),
+                               int(seg_rows), _ptr(S_x, torch.float32, "S_x"), _ptr(bias, torch.float32, "bias"),
+                               int(act), _ptr(Y, torch.float32, "Y"), M, N, K, _any_ptr(workspace, "workspace"),
+                               workspace.numel() * workspace.element_size(), _ptr(dbg_Xq, torch.int8, "dbg_Xq"),
+                               _ptr(dbg_acc, torch.int32, "dbg_acc"), _stream(stream))
+    _check(st, "q8_linear_wseg")
+    return Y
+
+
+def q8_linear_q_wseg(Xq, S_x, Wq, S_w, seg_rows: int, bias=None, act: int = Q8_ACT_NONE, Y=None, dbg_acc=None,
+                     dev_status=None, stream=None):
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float32, device=Xq.device)
+    st = load().q8_linear_q_wseg(_ptr(Xq, torch.int8, "Xq"), _ptr(S_x, torch.float32, "S_x"), _ptr(Wq, torch.int8, "Wq"),
+                                 _ptr(S_w, torch.float32, "S_w"), int(seg_rows), _ptr(bias, torch.float32, "bias"),
+                                 int(act), _ptr(Y, torch.float32, "Y"), M, N, K, _ptr(dbg_acc, torch.int32, "dbg_acc"),
+                                 _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
+    _check(st, "q8_linear_q_wseg")
+    return Y
 
 
 def q8_linear_requant(X, Wq, S_w, S_x, bias, act, S_y, Yq=None, Y=None, workspace=None, dbg_Xq=None, dbg_acc=None,

@@ -69,7 +69,7 @@ q8_status run_gemm(const GemmArgs &g, bool force_generic, cudaStream_t s)
 q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
                       float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
                       int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic, int8_t *Yq,
-                      const float *S_y)
+                      const float *S_y, int64_t w_seg)
 {
     last_launch_info() = LaunchInfo();
     q8_status st = check_gemm_shape(M, N, K);
@@ -79,6 +79,7 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
     if (!Y && !Yq) return Q8_ERR_NULL;
     if (Yq && !S_y) return Q8_ERR_NULL;
     if (S_y && !aligned_to(S_y, 4)) return Q8_ERR_ALIGN;
+    if (w_seg < 0) return Q8_ERR_SHAPE;
     if (act != Q8_ACT_NONE && act != Q8_ACT_GELU) return Q8_ERR_ARG;
     if (!aligned_to(X, 4) || !aligned_to(Y, 4) || !aligned_to(S_w, 4) || (S_x && !aligned_to(S_x, 4)) ||
         (bias && !aligned_to(bias, 4)) || (dbg_acc && !aligned_to(dbg_acc, 4)) || !aligned_to(workspace, 256))
@@ -99,6 +100,7 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
     g.Wq = Wq;
     g.S_x = S_x ? S_x : &hdr->S_x_dyn;
     g.S_w = S_w;
+    g.w_seg = w_seg;
     g.bias = bias;
     g.Y = Y;
     g.Yq = Yq;
@@ -156,6 +158,29 @@ q8_status q8_quantize_activation(const float *X, int64_t numel, const float *S_x
     return Q8_OK;
 }
 
+q8_status q8_fake_quantize(const float *X, int64_t numel, const float *S, float *Xhat, void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (numel < 0) return Q8_ERR_SHAPE;
+    if (numel == 0) return Q8_OK;
+    if (!X || !S || !Xhat) return Q8_ERR_NULL;
+    if (!aligned_to(X, 4) || !aligned_to(S, 4) || !aligned_to(Xhat, 4)) return Q8_ERR_ALIGN;
+    Q8_CUDA_TRY(launch_fake_quantize(X, numel, S, Xhat, static_cast<cudaStream_t>(stream)));
+    last_launch_info().launches = 1;
+    return Q8_OK;
+}
+
+q8_status q8_ste_backward(const float *grad_out, int64_t numel, float *grad_in, void *stream)
+{
+    last_launch_info() = LaunchInfo();
+    if (numel < 0) return Q8_ERR_SHAPE;
+    if (numel == 0 || grad_in == grad_out) return Q8_OK;  // the estimator is the identity: in place is a no-op
+    if (!grad_out || !grad_in) return Q8_ERR_NULL;
+    Q8_CUDA_TRY(cudaMemcpyAsync(grad_in, grad_out, (size_t)numel * sizeof(float), cudaMemcpyDeviceToDevice,
+                                static_cast<cudaStream_t>(stream)));
+    return Q8_OK;
+}
+
 size_t q8_calibrate_state_bytes(void) { return sizeof(CalibState); }
 
 q8_status q8_calibrate(const float *X, int64_t numel, float decay, void *state, void *stream)
@@ -200,7 +225,7 @@ q8_status q8_linear_generic(const float *X, const int8_t *Wq, const float *S_w, 
 // Body of q8_linear_q / q8_linear_q_requant.
 static q8_status linear_q_impl(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w,
                                const float *bias, int act, float *Y, int8_t *Yq, const float *S_y, int64_t M, int64_t N,
-                               int64_t K, int32_t *dbg_acc, int32_t *dev_status, void *stream)
+                               int64_t K, int32_t *dbg_acc, int32_t *dev_status, void *stream, int64_t w_seg = 0)
 {
     last_launch_info() = LaunchInfo();
     q8_status st = check_gemm_shape(M, N, K);
@@ -217,6 +242,7 @@ static q8_status linear_q_impl(const int8_t *Xq, const float *S_x, const int8_t 
     g.Wq = Wq;
     g.S_x = S_x;
     g.S_w = S_w;
+    g.w_seg = w_seg < 0 ? 0 : w_seg;
     g.bias = bias;
     g.Y = Y;
     g.Yq = Yq;
@@ -244,6 +270,42 @@ q8_status q8_linear_q_requant(const int8_t *Xq, const float *S_x, const int8_t *
 {
     if (M > 0 && N > 0 && !Yq) return Q8_ERR_NULL;
     return linear_q_impl(Xq, S_x, Wq, S_w, bias, act, Y, Yq, S_y, M, N, K, dbg_acc, dev_status, stream);
+}
+
+q8_status q8_quantize_weight_segments(const float *W, int64_t N, int64_t K, int64_t seg_rows, int8_t *Wq, float *S_w,
+                                      int32_t *dev_status, void *stream)
+{
+    if (seg_rows <= 0 || N < 0 || K < 0) return Q8_ERR_SHAPE;
+    int launches = 0;
+    for (int64_t r0 = 0, seg = 0; r0 < N; r0 += seg_rows, ++seg) {
+        const int64_t rows = (N - r0 < seg_rows) ? N - r0 : seg_rows;
+        q8_status st = q8_quantize_weight(W ? W + r0 * K : nullptr, rows, K, Wq ? Wq + r0 * K : nullptr,
+                                          S_w ? S_w + seg : nullptr, dev_status, stream);
+        if (st != Q8_OK) return st;
+        launches += last_launch_info().launches;
+    }
+    last_launch_info().launches = launches;
+    return Q8_OK;
+}
+
+q8_status q8_linear_wseg(const float *X, const int8_t *Wq, const float *S_w, int64_t w_seg_rows, const float *S_x,
+                         const float *bias, int act, float *Y, int64_t M, int64_t N, int64_t K, void *workspace,
+                         size_t workspace_bytes, int8_t *dbg_Xq, int32_t *dbg_acc, void *stream)
+{
+    if (w_seg_rows <= 0) return Q8_ERR_SHAPE;
+    if (M > 0 && N > 0 && !Y) return Q8_ERR_NULL;
+    return linear_impl(X, Wq, S_w, S_x, bias, act, Y, M, N, K, workspace, workspace_bytes, dbg_Xq, dbg_acc, stream, false,
+                       nullptr, nullptr, w_seg_rows);
+}
+
+q8_status q8_linear_q_wseg(const int8_t *Xq, const float *S_x, const int8_t *Wq, const float *S_w, int64_t w_seg_rows,
+                           const float *bias, int act, float *Y, int64_t M, int64_t N, int64_t K, int32_t *dbg_acc,
+                           int32_t *dev_status, void *stream)
+{
+    if (w_seg_rows <= 0) return Q8_ERR_SHAPE;
+    if (M > 0 && N > 0 && !Y) return Q8_ERR_NULL;
+    return linear_q_impl(Xq, S_x, Wq, S_w, bias, act, Y, nullptr, nullptr, M, N, K, dbg_acc, dev_status, stream,
+                         w_seg_rows);
 }
 
 q8_status q8_linear_requant(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias,

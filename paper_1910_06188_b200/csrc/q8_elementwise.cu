@@ -235,6 +235,32 @@ __global__ void __launch_bounds__(kThreads) embedding_kernel(const int32_t *__re
     }
 }
 
+// ------------------------------------------------------------------ training mode: fake quantisation (Sec. 2.2)
+// x_hat = Quantize(x | S) / S: the rounding of Eq. 1 simulated in floating point (one fp32 division per element).
+__device__ __forceinline__ float fake_one(float x, float S) { return __fdiv_rn((float)quantize_value(x, S), S); }
+
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads) fake_quantize_kernel(const float *__restrict__ x, int64_t n,
+                                                                 const float *__restrict__ S_ptr,
+                                                                 float *__restrict__ xhat)
+{
+    const float S = __ldg(S_ptr);
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    if (VEC) {
+        const float4 *x4 = reinterpret_cast<const float4 *>(x);
+        float4 *o4 = reinterpret_cast<float4 *>(xhat);
+        const int64_t n4 = n >> 2;
+        for (int64_t i = tid; i < n4; i += nthreads) {
+            const float4 v = __ldg(x4 + i);
+            o4[i] = make_float4(fake_one(v.x, S), fake_one(v.y, S), fake_one(v.z, S), fake_one(v.w, S));
+        }
+        for (int64_t j = (n4 << 2) + tid; j < n; j += nthreads) xhat[j] = fake_one(x[j], S);
+    } else {
+        for (int64_t j = tid; j < n; j += nthreads) xhat[j] = fake_one(x[j], S);
+    }
+}
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
@@ -263,6 +289,17 @@ cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *x
         quantize_kernel<true><<<grid_for((n + 3) >> 2, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy);
     } else {
         quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fake_quantize(const float *x, int64_t n, const float *S, float *xhat, cudaStream_t s)
+{
+    if (n <= 0) return cudaSuccess;
+    if (aligned16(x) && aligned16(xhat)) {
+        fake_quantize_kernel<true><<<grid_for((n + 3) >> 2, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xhat);
+    } else {
+        fake_quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xhat);
     }
     return cudaGetLastError();
 }

@@ -48,13 +48,14 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(GemmArgs a)
         __syncthreads();
     }
 
-    const float S_out = __fmul_rn(__ldg(a.S_x), __ldg(a.S_w));
-    const float inv = __fdiv_rn(1.0f, S_out);
+    const float S_x = __ldg(a.S_x);
     const float S_y = a.Yq ? __ldg(a.S_y) : 1.0f;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int64_t n = n0 + tx * 4 + j;
         if (n >= a.N) continue;
+        const float S_out = __fmul_rn(S_x, __ldg(a.S_w + (a.w_seg > 0 ? n / a.w_seg : 0)));
+        const float inv = __fdiv_rn(1.0f, S_out);
         const int32_t bq = a.bias ? quantize_bias(__ldg(a.bias + n), S_out) : 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

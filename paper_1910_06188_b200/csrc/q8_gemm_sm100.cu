@@ -289,7 +289,7 @@ __device__ __forceinline__ float gelu_fast(float y)
 template <int COLS, typename Release>
 __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
                                               uint32_t taddr, int64_t row0, int64_t col0, const int32_t (&bqv)[COLS / 32],
-                                              float inv, uint8_t *stage, int32_t *bq_s, int lane, Release release)
+                                              const float (&invv)[COLS / 32], uint8_t *stage, int32_t *bq_s, int lane, Release release)
 {
     constexpr int NCHUNK = COLS / 32;
     const int64_t row = row0 + lane;
@@ -299,6 +299,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
 #pragma unroll
     for (int ci = 0; ci < NCHUNK; ++ci) {
         const int64_t nb = col0 + 32 * ci;
+        const float inv = invv[ci];
         // b_q of these 32 columns (one per lane, computed before the accumulator was ready) -> all lanes
         __syncwarp();
         bq_s[lane] = bqv[ci];
@@ -527,8 +528,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32*quarter .. +31
         const int col_off = (ew >> 2) * C::kColsPerWarp;
         const bool active = col_off < BLOCK_N;
-        const float S_out = __fmul_rn(__ldg(a.S_x), __ldg(a.S_w));
-        const float inv = __fdiv_rn(1.0f, S_out);
+        const float S_x = __ldg(a.S_x);
+        // product scale S_x * S_w of the 32-column block starting at column n (w_seg is a multiple of 32 here,
+        // so a block never straddles two weight-scale segments)
+        auto product_scale = [&](int64_t n) {
+            const int64_t seg = (a.w_seg > 0 && n < a.N) ? n / a.w_seg : 0;
+            return __fmul_rn(S_x, __ldg(a.S_w + seg));
+        };
         uint8_t *stage = smem_stage + ew * kStagingBytesPerWarp;
         int32_t *bq_s = smem_bq + ew * 32;
         int as = 0;
@@ -553,7 +559,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             // b_q of this warp's columns (Sec. 3: bias quantised at S_x * S_w)
             int32_t bqv[NCH];
 #pragma unroll
-            for (int ci = 0; ci < NCH; ++ci) bqv[ci] = quantize_bias(bias_next[ci], S_out);
+            float invv[NCH];
+#pragma unroll
+            for (int ci = 0; ci < NCH; ++ci) {
+                const float S_out = product_scale(n0 + col_off + 32 * ci);
+                bqv[ci] = quantize_bias(bias_next[ci], S_out);
+                invv[ci] = __fdiv_rn(1.0f, S_out);
+            }
             fetch_bias(tile + num_units, bias_next);
             ok = mbar_wait(smem_u32(tmem_full_bar + as), aphase, abort_flag, a.status);
             ok = __all_sync(0xffffffffu, ok);
@@ -571,7 +583,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             if (active)
                 epilogue_warp<C::kColsPerWarp>(a, &tmap_y, tma_store != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
-                                               m0 + quarter * 32, n0 + col_off, bqv, inv, stage, bq_s, lane, release);
+                                               m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, release);
             else
                 release();
             if (++as == kAccStages) { as = 0; aphase ^= 1u; }
@@ -764,7 +776,8 @@ void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps)
 bool tcgen05_gemm_supported(const GemmArgs &a)
 {
     return (a.K % 16 == 0) && ((reinterpret_cast<uintptr_t>(a.Xq) & 15u) == 0) &&
-           ((reinterpret_cast<uintptr_t>(a.Wq) & 15u) == 0) && a.M < (int64_t(1) << 31) && a.N < (int64_t(1) << 31);
+           ((reinterpret_cast<uintptr_t>(a.Wq) & 15u) == 0) && a.M < (int64_t(1) << 31) && a.N < (int64_t(1) << 31) &&
+           (a.w_seg % 32 == 0);
 }
 
 cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s)

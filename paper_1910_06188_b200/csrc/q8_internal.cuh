@@ -30,7 +30,8 @@ struct GemmArgs {
     const int8_t *Xq;   // [M,K]
     const int8_t *Wq;   // [N,K]
     const float *S_x;   // device scalar
-    const float *S_w;   // device scalar
+    const float *S_w;   // device scalar, or one scale per block of w_seg output rows of W
+    int64_t w_seg = 0;  // rows of W (output features) that share one weight scale; 0 = one scale for all
     const float *bias;  // [N] or nullptr
     float *Y;           // [M,N] fp32 output, or nullptr when only the re-quantised output is wanted
     int8_t *Yq;         // [M,N] Int8 output Quantize(y | S_y) (Eq. 1 at the consumer's scale), or nullptr
@@ -59,6 +60,7 @@ cudaError_t launch_scale_from_absmax(const uint32_t *bits, float *S, int32_t *st
 cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy,
                             cudaStream_t s);
 cudaError_t launch_ema_update(CalibState *st, float decay, cudaStream_t s);
+cudaError_t launch_fake_quantize(const float *x, int64_t n, const float *S, float *xhat, cudaStream_t s);
 cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,
                              int64_t H, float *out, int8_t *rows_q, int32_t *status, cudaStream_t s);
 
@@ -79,7 +81,7 @@ cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_
 q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
                       float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
                       int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic, int8_t *Yq = nullptr,
-                      const float *S_y = nullptr);
+                      const float *S_y = nullptr, int64_t w_seg = 0);
 
 // Eq. 1 on one value: one rounded fp32 multiply, nearest-even integer (NaN -> 0, saturating), symmetric clamp.
 __device__ __forceinline__ int32_t quantize_value(float x, float S)

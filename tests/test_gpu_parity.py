@@ -254,3 +254,47 @@ def test_embedding_bad_ids_are_flagged_and_zeroed():
     got = out.cpu().numpy()
     assert not got[3].any() and not got[11].any()
     assert_close_fp(got, out_ref, "embedding with bad ids")
+
+
+# ------------------------------------------------------------------ training-mode pieces (Sec. 2.2, Eq. 5)
+@pytest.mark.parametrize("n", [1, 7, 4096, 100_003])
+def test_fake_quantize_and_ste(n):
+    x = synth.activation(1, n, seed=1300 + n).reshape(-1)
+    state = q8.new_calibrate_state()
+    q8.q8_calibrate(dev(x), 0.9, state)                       # the EMA update training does on every forward
+    S = q8.calibrate_S_x(state)
+    xh = q8.q8_fake_quantize(dev(x), S).cpu().numpy()
+    S_ref, _ = o.scale_from_absmax(o.absmax(x))
+    assert S.item() == S_ref
+    ref = o.fake_quantize(x, S_ref)
+    assert np.abs(xh - ref).max() <= 1e-6 * max(np.abs(ref).max(), 1e-30)
+    # the fake-quantised values sit exactly on the Int8 grid of the real quantiser
+    assert np.array_equal(np.rint(xh.astype(np.float64) * float(S_ref)).astype(np.int8), o.quantize(x, S_ref))
+    g = synth.normal((n,), 1.0, 1400 + n)
+    assert np.array_equal(q8.q8_ste_backward(dev(g)).cpu().numpy(), g)
+    gd = dev(g)
+    assert q8.q8_ste_backward(gd, gd).data_ptr() == gd.data_ptr()
+
+
+# ------------------------------------------------------------------ one weight scale per fused layer (Eq. 3 per layer)
+@pytest.mark.parametrize("M,H,seg,act", [(300, 128, 128, 0), (515, 256, 256, 1), (64, 40, 40, 0)])
+def test_fused_projection_with_per_layer_scales_equals_separate_layers(M, H, seg, act):
+    """Q, K and V stored as one [3H, H] matrix with one S_w per block of H rows must give what three separate
+    quantised FC layers give (the paper's model has three layers, each with its own Eq. 3 scale)."""
+    X = synth.activation(M, H, seed=1500 + M)
+    Ws = [synth.normal((H, H), 0.02 * (1 + 2 * i), 1501 + M + i) for i in range(3)]   # different ranges per layer
+    bs = [synth.bias(H, 1510 + M + i) for i in range(3)]
+    W, b = np.concatenate(Ws), np.concatenate(bs)
+    Wq, S_w = q8.q8_quantize_weight_segments(dev(W), seg)
+    acc = torch.empty((M, 3 * H), dtype=torch.int32, device="cuda")
+    Y = q8.q8_linear_wseg(dev(X), Wq, S_w, seg, None, dev(b), act, dbg_acc=acc)
+    info = q8.q8_last_launch_info()
+    assert info["gemm_kernel"] == (1 if seg % 32 == 0 else 2)
+    for i in range(3):
+        Wq_ref, S_ref, _ = o.quantize_weight(Ws[i])
+        assert S_w[i].item() == S_ref and np.array_equal(Wq[i * H:(i + 1) * H].cpu().numpy(), Wq_ref)
+        ref = o.linear(X, Wq_ref, S_ref, None, bs[i], act)
+        assert np.array_equal(acc[:, i * H:(i + 1) * H].cpu().numpy(), ref["acc"])
+        assert_close_fp(Y[:, i * H:(i + 1) * H].cpu().numpy(), ref["y"], f"segment {i}")
+    Xq, S_x = q8.q8_quantize_activation(dev(X))
+    assert torch.equal(q8.q8_linear_q_wseg(Xq, S_x, Wq, S_w, seg, dev(b), act), Y)

@@ -333,3 +333,24 @@ def test_attention_special_cases_and_numpy():
     # a single token attends to itself only
     one = rng.standard_normal((3, 3 * H)).astype(np.float32)
     assert np.allclose(o.attention(one, 3, 1, heads), one[:, 2 * H:], atol=0)
+
+
+# ---------------------------------------------------------------- training mode (Sec. 2.2, Eq. 5)
+def test_fake_quantize_grid_bound_and_idempotence(pins):
+    g = pins["dynamic_scale_example"]
+    xh = o.fake_quantize(np.array(g["x"], np.float32), g["S"])
+    assert np.allclose(xh, g["dequant"], rtol=0, atol=1e-15)            # the hand-worked dequantised values
+    rng = np.random.default_rng(61)
+    x = (rng.standard_normal(100_000) * 2).astype(np.float32)
+    S, _ = o.scale_from_absmax(o.absmax(x))
+    xh = o.fake_quantize(x, S)
+    assert np.abs(xh - x).max() <= 0.5 / float(S) * (1 + 1e-5)           # rounding error bound of Eq. 1
+    k = xh * float(S)
+    assert np.allclose(k, np.rint(k), atol=1e-9) and np.abs(np.rint(k)).max() == 127   # values sit on the Int8 grid
+    assert np.array_equal(o.fake_quantize(xh.astype(np.float32), S), xh)  # quantising a grid value changes nothing
+    assert np.array_equal(o.fake_quantize(-x, S), -xh)
+
+
+def test_straight_through_estimator_is_identity():
+    g = np.random.default_rng(63).standard_normal(1000).astype(np.float32)
+    assert np.array_equal(o.ste_backward(g), g.astype(np.float64))       # Eq. 5: gradient passes unchanged
