@@ -37,6 +37,10 @@ WORKLOADS = {
     "bert_large_fc": (4, synth.BERT_LARGE, "BERT-Large FC set, batch 64 x seq 384 (M=24576 tokens)"),
     "bert_base_fc": (2, synth.BERT_BASE, "BERT-Base FC set, batch 32 x seq 128 (M=4096 tokens)"),
 }
+# dram__bytes_read.sum + dram__bytes_write.sum of the tcgen05 GEMM per launch on the BERT-Large FC set, from the
+# ncu captures summarised in profiles/gemm_tcgen05_dram_traffic_m24576.md (one layer resident per capture).  Below the
+# algorithmic bytes because part of each output is still dirty in the 126 MB L2 when the kernel ends.
+GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 269279232, "attn_out": 66556416, "ffn1": 371026176, "ffn2": 163764480}}
 NOMINAL_INT8_OVER_BF16 = 2.0  # dense tensor peak ratio int8 : bf16 (4.5 : 2.25 POPS nominal)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -383,7 +387,10 @@ def run_ours(args):
     roofline = {
         "kernel": "gemm_tcgen05_kernel (4 launches per step, one per FC layer)",
         "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
-        "traffic": None,
+        "traffic": (sum(GEMM_DRAM_TRAFFIC[args.workload][L["name"]] for L in layers) / len(layers)
+                    if args.workload in GEMM_DRAM_TRAFFIC else None),
+        "traffic_note": "mean DRAM bytes per GEMM launch from ncu (profiles/gemm_tcgen05_dram_traffic_m24576.md); "
+                        "algorithmic mean is %.0f" % (sum(gemm_bytes) / len(gemm_bytes)),
         "peak_source": f"2 x {peak_key} of {peak_kind} (nominal int8:bf16 dense ratio); "
                        + ("burst figure: SM clock at max in the timed region" if at_max_clock else "sustained figure: SM clock below max"),
         "frac_of_sustained_peak": achieved / int8_peak_sustained,
