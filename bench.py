@@ -30,7 +30,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_1910_06188_b200 import synth  # noqa: E402
+from paper_1910_06188_b200 import dist_util, synth  # noqa: E402
 
 WORKLOADS = {
     # name: (config index, model dims, description)
@@ -198,7 +198,7 @@ def run_ours(args):
     cfg_index, dims, desc = WORKLOADS[args.workload]
     # weak scaling: every rank owns one full batch of M tokens (rows are independent given static
     # scales, so there is no data-path collective); rank r draws its batch from its own seeds.
-    M, layers = make_layers(cfg_index + 100 * rank, dims)
+    M, layers = make_layers(dist_util.rank_config(cfg_index, rank), dims)
     if args.layers:
         keep = set(args.layers.split(","))
         layers = [L for L in layers if L["name"] in keep]
@@ -221,7 +221,7 @@ def run_ours(args):
         del L["calib"], L["W"]
     E = synth.embedding_table(V, H, synth.seed_for(cfg_index, 90))
     Eq, S_e = q8.q8_quantize_weight(torch.from_numpy(E).to(dev))
-    ids = torch.from_numpy(synth.token_ids(M, V, synth.seed_for(cfg_index + 100 * rank, 91))).to(dev)
+    ids = torch.from_numpy(synth.token_ids(M, V, synth.seed_for(dist_util.rank_config(cfg_index, rank), 91))).to(dev)
     emb_out = torch.empty((M, H), dtype=torch.float32, device=dev)
     torch.cuda.synchronize()
 
@@ -315,12 +315,9 @@ def run_ours(args):
             dist.destroy_process_group()
         return 0
 
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = dist_util.max_over_ranks(ms, dev)
     ms_per_step = ms / args.steps
-    value = world * ops / (ms_per_step * 1e-3) / 1e12
+    value = dist_util.whole_job_rate(ops, world, ms_per_step) / 1e12
 
     # ---- end to end: host buffers, H2D of every input and D2H of every output inside the timed region
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -348,11 +345,8 @@ def run_ours(args):
     ev1.record(stream)
     barrier()
     e2e_ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * ops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_ms = dist_util.max_over_ranks(e2e_ms, dev)
+    e2e_value = dist_util.whole_job_rate(ops, world, e2e_ms / e2e_steps) / 1e12
 
     if rank != 0:
         if world > 1:
