@@ -30,7 +30,8 @@ def build(force: bool = False) -> str:
 def lib() -> C.CDLL:
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
+        # Q8_ORACLE_SO lets the mutation test point the pins at a deliberately broken build of the oracle
+        L = C.CDLL(os.environ.get("Q8_ORACLE_SO") or build())
         fp, i8p, i32p, dp = (C.POINTER(C.c_float), C.POINTER(C.c_int8), C.POINTER(C.c_int32),
                              C.POINTER(C.c_double))
         ip = C.POINTER(C.c_int)
