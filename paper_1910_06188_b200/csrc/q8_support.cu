@@ -93,7 +93,8 @@ __global__ void __launch_bounds__(256) attention_kernel(const float *__restrict_
     const int64_t row_pitch = 3 * H;
     const float *base = qkv + seq * S * row_pitch + head * kD;
 
-    // queries of this CTA (pre-scaled), transposed; rows past the sequence end are zero
+    // queries of this CTA, pre-scaled by log2(e) / sqrt(d) so that the softmax can use exp2 directly, transposed;
+    // rows past the sequence end are zero
     for (int e = threadIdx.x; e < kTile * kD; e += 256) {
         const int i = e / kD, d = e % kD;
         Qt[d][i] = (q0 + i < S) ? base[(q0 + i) * row_pitch + d] * scale : 0.0f;
@@ -107,15 +108,31 @@ __global__ void __launch_bounds__(256) attention_kernel(const float *__restrict_
         l[a] = 0.0f;
     }
 
-    for (int64_t j0 = 0; j0 < S; j0 += kTile) {
-        __syncthreads();  // previous tile fully consumed (and Qt written, on the first pass)
-        for (int e = threadIdx.x; e < kTile * kD; e += 256) {
+    // The next key / value tile is fetched into registers while the current one is being used, so the global
+    // load latency overlaps the arithmetic.  Element e = tid + 256 i of a tile is (key j = e / 64, feature d = e % 64).
+    float kreg[16], vreg[16];
+    auto fetch_tile = [&](int64_t j0) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int e = threadIdx.x + 256 * i;
             const int j = e / kD, d = e % kD;
             const bool ok = j0 + j < S;
-            Kt[d][j] = ok ? base[(j0 + j) * row_pitch + H + d] : 0.0f;
-            Vs[j][d] = ok ? base[(j0 + j) * row_pitch + 2 * H + d] : 0.0f;
+            kreg[i] = ok ? __ldg(base + (j0 + j) * row_pitch + H + d) : 0.0f;
+            vreg[i] = ok ? __ldg(base + (j0 + j) * row_pitch + 2 * H + d) : 0.0f;
+        }
+    };
+    fetch_tile(0);
+
+    for (int64_t j0 = 0; j0 < S; j0 += kTile) {
+        __syncthreads();  // previous tile fully consumed (and Qt written, on the first pass)
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int e = threadIdx.x + 256 * i;
+            Kt[e % kD][e / kD] = kreg[i];
+            Vs[e / kD][e % kD] = vreg[i];
         }
         __syncthreads();
+        if (j0 + kTile < S) fetch_tile(j0 + kTile);
 
         float s[4][4] = {};
 #pragma unroll 8
@@ -144,11 +161,11 @@ __global__ void __launch_bounds__(256) attention_kernel(const float *__restrict_
 #pragma unroll
             for (int off = 8; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
             const float m_new = fmaxf(m[a], mx);
-            const float corr = expf(m[a] - m_new);  // exp(-inf) = 0 on the first tile
+            const float corr = exp2f(m[a] - m_new);  // 2^(-inf) = 0 on the first tile
             float sum = 0.0f;
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
-                s[a][b] = expf(s[a][b] - m_new);
+                s[a][b] = exp2f(s[a][b] - m_new);
                 sum += s[a][b];
             }
 #pragma unroll
@@ -229,7 +246,7 @@ cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t hea
         attr_set[dev] = true;
     }
     dim3 grid((unsigned)((S + kTile - 1) / kTile), (unsigned)heads, (unsigned)B);
-    attention_kernel<<<grid, 256, kAttnSmemBytes, s>>>(qkv, S, heads * kD, 1.0f / 8.0f, ctx, S_q, ctx_q);
+    attention_kernel<<<grid, 256, kAttnSmemBytes, s>>>(qkv, S, heads * kD, 1.4426950408889634f / 8.0f, ctx, S_q, ctx_q);
     return cudaGetLastError();
 }
 
