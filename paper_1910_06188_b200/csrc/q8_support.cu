@@ -66,6 +66,125 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_kernel(const float *
     }
 }
 
+// Vector form for H % 4 == 0, H <= 4096 and 16-byte aligned rows: the row lives in registers (up to four
+// float4 per thread), every access is a 16-byte one, and the Int8 copy is written four values at a time.
+__global__ void __launch_bounds__(kLnThreads) add_layernorm_vec_kernel(const float *__restrict__ x,
+                                                                       const float *__restrict__ r1,
+                                                                       const float *__restrict__ r2,
+                                                                       const float *__restrict__ gamma,
+                                                                       const float *__restrict__ beta, float eps,
+                                                                       int64_t H, float *__restrict__ out,
+                                                                       const float *__restrict__ S_q,
+                                                                       int8_t *__restrict__ out_q)
+{
+    __shared__ float scratch[kLnThreads / 32];
+    const int64_t base4 = (int64_t)blockIdx.x * (H >> 2);
+    const int n4 = (int)(H >> 2);
+    const float4 *x4 = reinterpret_cast<const float4 *>(x) + base4;
+    const float4 *a4 = r1 ? reinterpret_cast<const float4 *>(r1) + base4 : nullptr;
+    const float4 *b4 = r2 ? reinterpret_cast<const float4 *>(r2) + base4 : nullptr;
+    float4 v[4];
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = threadIdx.x + kLnThreads * i;
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < n4) {
+            v[i] = x4[c];
+            if (a4) { const float4 t = a4[c]; v[i].x += t.x; v[i].y += t.y; v[i].z += t.z; v[i].w += t.w; }
+            if (b4) { const float4 t = b4[c]; v[i].x += t.x; v[i].y += t.y; v[i].z += t.z; v[i].w += t.w; }
+            s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+        }
+    }
+    const float mean = block_sum(s, scratch) / (float)H;
+    float q = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        if (threadIdx.x + kLnThreads * i < n4) {
+            const float dx = v[i].x - mean, dy = v[i].y - mean, dz = v[i].z - mean, dw = v[i].w - mean;
+            q += (dx * dx + dy * dy) + (dz * dz + dw * dw);
+        }
+    const float var = block_sum(q, scratch) / (float)H;
+    const float rstd = 1.0f / sqrtf(var + eps);
+    const float Sq = out_q ? __ldg(S_q) : 1.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = threadIdx.x + kLnThreads * i;
+        if (c >= n4) continue;
+        const float4 g = gamma ? reinterpret_cast<const float4 *>(gamma)[c] : make_float4(1.f, 1.f, 1.f, 1.f);
+        const float4 b = beta ? reinterpret_cast<const float4 *>(beta)[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 y;
+        y.x = (v[i].x - mean) * rstd * g.x + b.x;
+        y.y = (v[i].y - mean) * rstd * g.y + b.y;
+        y.z = (v[i].z - mean) * rstd * g.z + b.z;
+        y.w = (v[i].w - mean) * rstd * g.w + b.w;
+        if (out) reinterpret_cast<float4 *>(out)[base4 + c] = y;
+        if (out_q) reinterpret_cast<uint32_t *>(out_q)[base4 + c] = quantize_pack4(y.x, y.y, y.z, y.w, Sq);
+    }
+}
+
+// One warp per row for H <= 1024 (BERT's hidden sizes): up to eight float4 per lane, both moments reduced with
+// shuffles only, eight rows per CTA, so there is no block-level barrier at all.
+__global__ void __launch_bounds__(kLnThreads) add_layernorm_warp_kernel(const float *__restrict__ x,
+                                                                        const float *__restrict__ r1,
+                                                                        const float *__restrict__ r2,
+                                                                        const float *__restrict__ gamma,
+                                                                        const float *__restrict__ beta, float eps,
+                                                                        int64_t rows, int64_t H, float *__restrict__ out,
+                                                                        const float *__restrict__ S_q,
+                                                                        int8_t *__restrict__ out_q)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (kLnThreads / 32) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int n4 = (int)(H >> 2);
+    const int64_t base4 = row * n4;
+    const float4 *x4 = reinterpret_cast<const float4 *>(x) + base4;
+    const float4 *a4 = r1 ? reinterpret_cast<const float4 *>(r1) + base4 : nullptr;
+    const float4 *b4 = r2 ? reinterpret_cast<const float4 *>(r2) + base4 : nullptr;
+    float4 v[8];
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int c = lane + 32 * i;
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < n4) {
+            v[i] = __ldg(x4 + c);
+            if (a4) { const float4 t = __ldg(a4 + c); v[i].x += t.x; v[i].y += t.y; v[i].z += t.z; v[i].w += t.w; }
+            if (b4) { const float4 t = __ldg(b4 + c); v[i].x += t.x; v[i].y += t.y; v[i].z += t.z; v[i].w += t.w; }
+            s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const float mean = s / (float)H;
+    float q = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        if (lane + 32 * i < n4) {
+            const float dx = v[i].x - mean, dy = v[i].y - mean, dz = v[i].z - mean, dw = v[i].w - mean;
+            q += (dx * dx + dy * dy) + (dz * dz + dw * dw);
+        }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    const float rstd = 1.0f / sqrtf(q / (float)H + eps);
+    const float Sq = out_q ? __ldg(S_q) : 1.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int c = lane + 32 * i;
+        if (c >= n4) continue;
+        const float4 g = gamma ? __ldg(reinterpret_cast<const float4 *>(gamma) + c) : make_float4(1.f, 1.f, 1.f, 1.f);
+        const float4 b = beta ? __ldg(reinterpret_cast<const float4 *>(beta) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 y;
+        y.x = (v[i].x - mean) * rstd * g.x + b.x;
+        y.y = (v[i].y - mean) * rstd * g.y + b.y;
+        y.z = (v[i].z - mean) * rstd * g.z + b.z;
+        y.w = (v[i].w - mean) * rstd * g.w + b.w;
+        if (out) reinterpret_cast<float4 *>(out)[base4 + c] = y;
+        if (out_q) reinterpret_cast<uint32_t *>(out_q)[base4 + c] = quantize_pack4(y.x, y.y, y.z, y.w, Sq);
+    }
+}
+
 // ------------------------------------------------------------------ self-attention, head dimension 64, no mask
 // ctx[b, i, head] = softmax_j(q_i . k_j / 8) v_j with q, k, v read from the fused projection
 // qkv[T, 3H] = [q | k | v].  One CTA per (64 queries, head, sequence); keys and values stream through
@@ -226,8 +345,18 @@ cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r
                                  int8_t *out_q, cudaStream_t s)
 {
     if (rows <= 0 || H <= 0) return cudaSuccess;
-    add_layernorm_kernel<<<(unsigned)rows, kLnThreads, (size_t)H * sizeof(float), s>>>(x, r1, r2, gamma, beta, eps, H,
-                                                                                       out, S_q, out_q);
+    auto al16 = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+    const bool vec = (H % 4 == 0) && H <= 4 * 4 * kLnThreads && al16(x) && al16(r1) && al16(r2) && al16(gamma) &&
+                     al16(beta) && al16(out) && (reinterpret_cast<uintptr_t>(out_q) & 3u) == 0;
+    if (vec && H <= 1024) {
+        const unsigned blocks = (unsigned)((rows + kLnThreads / 32 - 1) / (kLnThreads / 32));
+        add_layernorm_warp_kernel<<<blocks, kLnThreads, 0, s>>>(x, r1, r2, gamma, beta, eps, rows, H, out, S_q, out_q);
+    } else if (vec) {
+        add_layernorm_vec_kernel<<<(unsigned)rows, kLnThreads, 0, s>>>(x, r1, r2, gamma, beta, eps, H, out, S_q, out_q);
+    } else {
+        add_layernorm_kernel<<<(unsigned)rows, kLnThreads, (size_t)H * sizeof(float), s>>>(x, r1, r2, gamma, beta, eps,
+                                                                                           H, out, S_q, out_q);
+    }
     return cudaGetLastError();
 }
 
