@@ -223,6 +223,17 @@ void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *gri
  * SMs per 256 x 256 tile).  Results do not depend on the choice.  Not thread-safe. */
 q8_status q8_tune_gemm_tile(int block_n, int ctas);
 
+/* Tuning / test hook for the schedule of the cta_group::2 kernel.  When the number of 256 x 256 tiles
+ * is not a multiple of the number of SM pairs, the tiles of the last, partial round are cut into 2 or 4
+ * narrower tiles (256 x 128 or 256 x 64) if these still fit in one round, which shortens that round.
+ * enable = 0 switches this off for later calls in this process, non-zero (the default) on.  Results do
+ * not depend on it.  Not thread-safe.  (An implementation detail with no counterpart in the paper.) */
+void q8_tune_gemm_tail_split(int enable);
+
+/* Into how many narrower tiles each tile of the last round was cut by the most recent tcgen05 GEMM launch
+ * of this host thread: 1 (not cut), 2 or 4. */
+int q8_last_launch_tail_split(void);
+
 #ifdef __cplusplus
 }
 #endif

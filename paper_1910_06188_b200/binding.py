@@ -49,6 +49,8 @@ SIGNATURES = {
     "q8_status_string": (C.c_char_p, [_int]),
     "q8_last_launch_info": (None, [C.POINTER(_int)] * 5),
     "q8_tune_gemm_tile": (_int, [_int, _int]),
+    "q8_tune_gemm_tail_split": (None, [_int]),
+    "q8_last_launch_tail_split": (_int, []),
 }
 
 _lib: Optional[C.CDLL] = None
@@ -426,6 +428,16 @@ def q8_last_launch_info() -> dict:
     a, b, c, d, e = C.c_int(0), C.c_int(0), C.c_int(0), C.c_int(0), C.c_int(0)
     load().q8_last_launch_info(C.byref(a), C.byref(b), C.byref(c), C.byref(d), C.byref(e))
     return dict(gemm_kernel=a.value, launches=b.value, block_n=c.value, grid=d.value, ctas=e.value)
+
+
+def q8_tune_gemm_tail_split(enable: bool = True) -> None:
+    """Switches the cutting of the last scheduling round's tiles into narrower ones on or off."""
+    load().q8_tune_gemm_tail_split(1 if enable else 0)
+
+
+def q8_last_launch_tail_split() -> int:
+    """1, 2 or 4: how many narrower tiles each last-round tile of the latest tcgen05 GEMM was cut into."""
+    return int(load().q8_last_launch_tail_split())
 
 
 def q8_tune_gemm_tile(block_n: int = 0, ctas: int = 0) -> None:

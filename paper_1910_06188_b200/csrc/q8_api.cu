@@ -446,4 +446,8 @@ q8_status q8_tune_gemm_tile(int block_n, int ctas)
     return Q8_OK;
 }
 
+void q8_tune_gemm_tail_split(int enable) { set_gemm_tail_split(enable != 0); }
+
+int q8_last_launch_tail_split(void) { return last_launch_info().tail_split; }
+
 }  // extern "C"

@@ -289,15 +289,17 @@ __device__ __forceinline__ float gelu_fast(float y)
 template <int COLS, typename Release>
 __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
                                               uint32_t taddr, int64_t row0, int64_t col0, const int32_t (&bqv)[COLS / 32],
-                                              const float (&invv)[COLS / 32], uint8_t *stage, int32_t *bq_s, int lane, Release release)
+                                              const float (&invv)[COLS / 32], uint8_t *stage, int32_t *bq_s, int lane, int nch,
+                                              Release release)
 {
-    constexpr int NCHUNK = COLS / 32;
+    constexpr int NCHUNK = COLS / 32;  // compile-time maximum; this tile has nch <= NCHUNK blocks (warp-uniform)
     const int64_t row = row0 + lane;
     const bool row_ok = row < a.M;
     const float S_y = a.Yq != nullptr ? __ldg(a.S_y) : 1.0f;
     const bool yq_vec = ((a.N & 15) == 0) && ((reinterpret_cast<uintptr_t>(a.Yq) & 15u) == 0);
 #pragma unroll
     for (int ci = 0; ci < NCHUNK; ++ci) {
+        if (ci >= nch) break;
         const int64_t nb = col0 + 32 * ci;
         const float inv = invv[ci];
         // b_q of these 32 columns (one per lane, computed before the accumulator was ready) -> all lanes
@@ -307,7 +309,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
         uint32_t v[32];
         tmem_ld_32x32(taddr + (uint32_t)(32 * ci), v);
         tmem_ld_wait();
-        if (ci + 1 == NCHUNK) release();
+        if (ci + 1 == nch) release();
         if (nb >= a.N || row0 >= a.M) continue;  // warp-uniform: the block lies outside the matrix
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
@@ -378,7 +380,8 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
 template <int BLOCK_N, int CTAS, int EW>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                    const __grid_constant__ CUtensorMap tmap_y, GemmArgs a, int tma_store)
+                    const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_w4,
+                    const __grid_constant__ CUtensorMap tmap_y, GemmArgs a, int tma_store, int64_t full_tiles, int split)
 {
     using C = Cfg<BLOCK_N, CTAS, EW>;
     constexpr int kEpilogueWarps = EW;
@@ -403,7 +406,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const int64_t unit = blockIdx.x / CTAS, num_units = gridDim.x / CTAS;  // a unit = one CTA or one CTA pair
     const int64_t tiles_n = (a.N + BLOCK_N - 1) / BLOCK_N;
     const int64_t tiles_m = (a.M + TILE_M - 1) / TILE_M;
-    const int64_t num_tiles = tiles_m * tiles_n;
+    // Tile schedule.  Tiles [0, full_tiles) are whole BLOCK_N-wide tiles and fill complete rounds over the
+    // units; the leftover tiles of the last, partial round are cut into `split` narrower tiles each (same rows,
+    // BLOCK_N / split columns), so that the tail keeps more units busy for a shorter time.
+    const int64_t num_tiles = full_tiles + (tiles_m * tiles_n - full_tiles) * split;
+    const int32_t tiles_n32 = (int32_t)tiles_n, full32 = (int32_t)full_tiles;  // tile counts fit 32 bits by far
+    auto decode = [&](int64_t t, int64_t &m_idx, int64_t &n0, int &width) {
+        int32_t whole = (int32_t)t, sub = 0;
+        width = BLOCK_N;
+        if (whole >= full32) {
+            const int32_t u = whole - full32;
+            width = BLOCK_N / split;
+            whole = full32 + u / split;
+            sub = u % split;
+        }
+        const int32_t mi = whole / tiles_n32;
+        m_idx = mi;
+        n0 = (whole - mi * tiles_n32) * BLOCK_N + sub * width;
+    };
     const int num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
 
     if (threadIdx.x == 0) {
@@ -436,23 +456,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             int issued = 0;
             bool ok = true;
             for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
-                const int32_t m0 = (int32_t)((tile / tiles_n) * TILE_M + cta_rank * BLOCK_M);
-                const int32_t n0 = (int32_t)((tile % tiles_n) * BLOCK_N + cta_rank * C::kBRows);
+                int64_t m_idx, n_start;
+                int width;
+                decode(tile, m_idx, n_start, width);
+                const int b_rows = width / CTAS;  // W_q rows this CTA loads for the tile
+                const int32_t m0 = (int32_t)(m_idx * TILE_M + cta_rank * BLOCK_M);
+                const int32_t n0 = (int32_t)(n_start + cta_rank * b_rows);
+                const CUtensorMap *map_w = width == BLOCK_N ? &tmap_w : (width * 2 == BLOCK_N ? &tmap_w2 : &tmap_w4);
+                const uint32_t stage_bytes = (uint32_t)(C::kABytes + b_rows * BLOCK_K);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(smem_u32(empty_bar + s), phase ^ 1u, abort_flag, a.status);
                     if (!ok) break;
                     const uint32_t fb = smem_u32(full_bar + s);
                     const uint32_t dst_a = smem_u32(smem_a + s * C::kABytes), dst_b = smem_u32(smem_b + s * C::kBBytes);
                     if (CTAS == 1) {
-                        mbar_expect_tx(fb, C::kStageBytes);
+                        mbar_expect_tx(fb, stage_bytes);
                         tma_load_2d(dst_a, &tmap_x, kb * BLOCK_K, m0, fb);
-                        tma_load_2d(dst_b, &tmap_w, kb * BLOCK_K, n0, fb);
+                        tma_load_2d(dst_b, map_w, kb * BLOCK_K, n0, fb);
                     } else {
                         // both CTAs report their bytes to the leader's barrier, which the MMA warp waits on
-                        if (leader) mbar_expect_tx(fb, 2 * C::kStageBytes);
+                        if (leader) mbar_expect_tx(fb, 2 * stage_bytes);
                         const uint32_t fb_leader = map_to_cta(fb, 0);
                         tma_load_2d_pair(dst_a, &tmap_x, kb * BLOCK_K, m0, fb_leader);
-                        tma_load_2d_pair(dst_b, &tmap_w, kb * BLOCK_K, n0, fb_leader);
+                        tma_load_2d_pair(dst_b, map_w, kb * BLOCK_K, n0, fb_leader);
                     }
                     ++issued;
                     if (++s == C::kStages) { s = 0; phase ^= 1u; }
@@ -489,6 +515,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(as * BLOCK_N);
+                // a narrow tile of the split tail runs the same MMA with a smaller N field (bits 17..22 = N / 8)
+                const uint32_t width = tile < full_tiles ? (uint32_t)BLOCK_N : (uint32_t)(BLOCK_N / split);
+                const uint32_t idesc = (C::kInstrDesc & ~(0x3Fu << 17)) | ((width >> 3) << 17);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(smem_u32(full_bar + s), phase, abort_flag, a.status);
                     if (!ok) break;
@@ -499,8 +528,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                         // +32 bytes along K inside the swizzle span == +2 in the (addr >> 4) field
                         const uint64_t adv = (uint64_t)(k * (UMMA_K >> 4));
-                        if (CTAS == 2) umma_i8_pair(tmem_d, da + adv, db + adv, C::kInstrDesc, (uint32_t)((kb | k) != 0));
-                        else umma_i8(tmem_d, da + adv, db + adv, C::kInstrDesc, (uint32_t)((kb | k) != 0));
+                        if (CTAS == 2) umma_i8_pair(tmem_d, da + adv, db + adv, idesc, (uint32_t)((kb | k) != 0));
+                        else umma_i8(tmem_d, da + adv, db + adv, idesc, (uint32_t)((kb | k) != 0));
                     }
                     // frees the stage (in both CTAs) once these MMAs have read it
                     if (CTAS == 2) umma_commit_pair(smem_u32(empty_bar + s));
@@ -526,8 +555,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // ---------------- epilogue ----------------
         const int ew = warp - 2;       // 0 .. 7
         const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32*quarter .. +31
-        const int col_off = (ew >> 2) * C::kColsPerWarp;
-        const bool active = col_off < BLOCK_N;
+        const int col_group = ew >> 2;  // which share of the tile's columns this warp takes
         const float S_x = __ldg(a.S_x);
         // product scale S_x * S_w of the 32-column block starting at column n (w_seg is a multiple of 32 here,
         // so a block never straddles two weight-scale segments)
@@ -544,21 +572,31 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         // global load takes microseconds, which would otherwise be exposed at the start of every tile.
         constexpr int NCH = C::kColsPerWarp / 32;
         float bias_next[NCH];
+        // Columns of a tile of `width` columns are shared out in equal runs of at least 32: warp group g takes
+        // [g * cpw, (g + 1) * cpw); on a narrow tile the groups past the end have nothing to do.
+        auto cols_per_warp = [&](int width) { return max(32, width / (EW / 4)); };
         auto fetch_bias = [&](int64_t tile, float (&dst)[NCH]) {
-            const int64_t n0 = (tile % tiles_n) * BLOCK_N;
+            int64_t m_idx, n0;
+            int width = BLOCK_N;
+            if (tile < num_tiles) decode(tile, m_idx, n0, width);
+            else n0 = a.N;
+            const int cpw = cols_per_warp(width), col_off = col_group * cpw;
 #pragma unroll
             for (int ci = 0; ci < NCH; ++ci) {
                 const int64_t n = n0 + col_off + 32 * ci + lane;
-                dst[ci] = (active && a.bias != nullptr && tile < num_tiles && n < a.N) ? __ldg(a.bias + n) : 0.0f;
+                dst[ci] = (col_off < width && 32 * ci < cpw && a.bias != nullptr && n < a.N) ? __ldg(a.bias + n) : 0.0f;
             }
         };
         fetch_bias(unit, bias_next);
         for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
-            const int64_t m0 = (tile / tiles_n) * TILE_M + cta_rank * BLOCK_M;
-            const int64_t n0 = (tile % tiles_n) * BLOCK_N;
+            int64_t m_idx, n0;
+            int width;
+            decode(tile, m_idx, n0, width);
+            const int64_t m0 = m_idx * TILE_M + cta_rank * BLOCK_M;
+            const int cpw = cols_per_warp(width), col_off = col_group * cpw;
+            const bool active = col_off < width;
             // b_q of this warp's columns (Sec. 3: bias quantised at S_x * S_w)
             int32_t bqv[NCH];
-#pragma unroll
             float invv[NCH];
 #pragma unroll
             for (int ci = 0; ci < NCH; ++ci) {
@@ -583,7 +621,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             if (active)
                 epilogue_warp<C::kColsPerWarp>(a, &tmap_y, tma_store != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
-                                               m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, release);
+                                               m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release);
             else
                 release();
             if (++as == kAccStages) { as = 0; aphase ^= 1u; }
@@ -668,6 +706,7 @@ int sm_count()
 
 int g_force_block_n = 0, g_force_ctas = 0;  // set by q8_tune_gemm_tile(); 0 = choose automatically
 int g_force_epilogue_warps = 0;            // 0 automatic, else 8 or 16 (cta_group::2 kernel only)
+bool g_tail_split_enabled = true;          // cut the tiles of a partial last round into narrower ones
 
 template <int BLOCK_N, int CTAS, int EW = 8>
 cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
@@ -706,9 +745,27 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
         max_units[dev] = units;
         attr_set[dev] = true;
     }
-    CUtensorMap tx, tw, ty;
+    const int64_t tiles = ((a.M + BLOCK_M * CTAS - 1) / (BLOCK_M * CTAS)) * ((a.N + BLOCK_N - 1) / BLOCK_N);
+    const int units = (int)(tiles < max_units[dev] ? tiles : max_units[dev]);
+    // Tail of the schedule: when the last round would leave most units idle, its tiles are cut into 2 or 4
+    // narrower ones (as many as still fit in one round), so the round is shorter by the saved W traffic and MMAs.
+    int split = 1;
+    int64_t full_tiles = tiles;
+    if (CTAS == 2 && g_tail_split_enabled && tiles > units && tiles % units != 0) {
+        const int64_t rest = tiles % units;
+        split = rest * 4 <= units ? 4 : (rest * 2 <= units ? 2 : 1);
+        if (split > 1) full_tiles = tiles - rest;
+    }
+    CUtensorMap tx, tw, tw2, tw4, ty;
     if (!make_tmap(&tx, a.Xq, a.M, a.K, BLOCK_M) || !make_tmap(&tw, a.Wq, a.N, a.K, C::kBRows))
         return cudaErrorInvalidValue;
+    if (split > 1) {
+        if (!make_tmap(&tw2, a.Wq, a.N, a.K, C::kBRows / 2) || !make_tmap(&tw4, a.Wq, a.N, a.K, C::kBRows / 4))
+            return cudaErrorInvalidValue;
+    } else {
+        tw2 = tw;  // never used
+        tw4 = tw;
+    }
     // the TMA store needs a 16-byte aligned base and row pitch; otherwise lanes store their rows directly
     int tma_store = a.Y != nullptr && ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
     if (tma_store) {
@@ -716,8 +773,6 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     } else {
         ty = tx;  // never dereferenced
     }
-    const int64_t tiles = ((a.M + BLOCK_M * CTAS - 1) / (BLOCK_M * CTAS)) * ((a.N + BLOCK_N - 1) / BLOCK_N);
-    const int units = (int)(tiles < max_units[dev] ? tiles : max_units[dev]);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(units * CTAS));
     cfg.blockDim = dim3(kThreads);
@@ -730,13 +785,14 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, kernel, tx, tw, ty, a, tma_store);
+    e = cudaLaunchKernelEx(&cfg, kernel, tx, tw, tw2, tw4, ty, a, tma_store, full_tiles, split);
     LaunchInfo &li = last_launch_info();
     li.gemm_kernel = 1;
     li.block_n = BLOCK_N;
     li.ctas = CTAS;
     li.epilogue_warps = EW;
     li.grid = units * CTAS;
+    li.tail_split = split;
     li.launches += 1;
     return e;
 }
@@ -772,6 +828,8 @@ void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps)
     g_force_ctas = ctas;
     g_force_epilogue_warps = epilogue_warps;
 }
+
+void set_gemm_tail_split(bool enable) { g_tail_split_enabled = enable; }
 
 bool tcgen05_gemm_supported(const GemmArgs &a)
 {

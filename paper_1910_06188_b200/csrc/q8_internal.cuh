@@ -49,6 +49,7 @@ struct LaunchInfo {
     int ctas = 0;  // CTAs cooperating on one tile (1, or 2 for cta_group::2)
     int epilogue_warps = 0;
     int grid = 0;
+    int tail_split = 1;  // tiles of the last scheduling round cut into this many narrower ones
 };
 LaunchInfo &last_launch_info();
 
@@ -74,6 +75,7 @@ cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t hea
 // ---- GEMM launchers ----
 bool tcgen05_gemm_supported(const GemmArgs &a);
 void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps = 0);  // 0, 0 = automatic choice
+void set_gemm_tail_split(bool enable);
 cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s);  // q8_gemm_sm100.cu
 cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_generic.cu
 

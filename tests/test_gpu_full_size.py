@@ -94,6 +94,31 @@ def test_every_tile_shape_matches_the_oracle(block_n, ctas):
         q8.q8_tune_gemm_tile(48, 1)
 
 
+@pytest.mark.parametrize("M,N,K,act", [(20000, 1000, 128, 1), (19463, 1088, 160, 0), (21000, 520, 144, 1)])
+def test_split_tail_of_the_pair_schedule_matches_the_oracle(M, N, K, act):
+    """Shapes whose 256 x 256 tiles do not fill the last round over the SM pairs: the tail is cut into
+    narrower tiles (ragged in M, N and K here), and the result is the oracle's either way."""
+    from tests.gpu_util import check_linear
+    X = synth.activation(M, K, seed=1200 + N)
+    W = synth.weight(N, K, seed=1201 + N)
+    bb = synth.bias(N, seed=1202 + N)
+    tiles = -(-M // 256) * -(-N // 256)
+    try:
+        q8.q8_tune_gemm_tile(256, 2)
+        info = check_linear(X, W, bb, act=act)
+        assert (info["block_n"], info["ctas"]) == (256, 2)
+        units = info["grid"] // 2  # SM pairs the launch ran on
+        rest = tiles % units
+        expect = 1 if (tiles <= units or rest == 0) else (4 if rest * 4 <= units else (2 if rest * 2 <= units else 1))
+        assert q8.q8_last_launch_tail_split() == expect
+        q8.q8_tune_gemm_tail_split(False)
+        check_linear(X, W, bb, act=act)
+        assert q8.q8_last_launch_tail_split() == 1
+    finally:
+        q8.q8_tune_gemm_tail_split(True)
+        q8.q8_tune_gemm_tile(0, 0)
+
+
 def test_empty_problem_is_a_noop():
     Wq = torch.ones((8, 16), dtype=torch.int8, device="cuda")
     S = torch.ones(1, device="cuda")
