@@ -234,6 +234,18 @@ void q8_tune_gemm_tail_split(int enable);
  * of this host thread: 1 (not cut), 2 or 4. */
 int q8_last_launch_tail_split(void);
 
+/* Measurement aid, no counterpart in the paper: the issue-bound Int8 rate of the tensor cores of the current
+ * device, i.e. the ceiling of the GEMM's tensor pipe when operands cost nothing.  Every SM (ctas = 1) or SM
+ * pair (ctas = 2, cta_group::2) issues the GEMM kernel's own tcgen05.mma kind::i8 shape (M = 128 * ctas,
+ * N = 256, K = 32) back to back on operand tiles that stay in shared memory (pseudo-random bytes; no TMA, no
+ * stores) for about `seconds` (0 < seconds <= 5; a short calibration launch sizes the timed launch).
+ * Host outputs: *tops = 2 M N K * instructions / time in 1e12 op/s (required), *elapsed_ms and *sms_used
+ * (either may be NULL).  `dev_status` (device int32, may be NULL) receives Q8_ERR_TIMEOUT bits should a wait
+ * inside the kernel give up.  Synchronises `stream`.  Returns Q8_ERR_ARG on bad arguments, Q8_ERR_CUDA when a
+ * runtime call fails. */
+q8_status q8_measure_int8_mma_peak(int ctas, double seconds, double *tops, double *elapsed_ms, int *sms_used,
+                                   void *dev_status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -51,6 +51,8 @@ SIGNATURES = {
     "q8_tune_gemm_tile": (_int, [_int, _int]),
     "q8_tune_gemm_tail_split": (None, [_int]),
     "q8_last_launch_tail_split": (_int, []),
+    "q8_measure_int8_mma_peak": (_int, [_int, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_int),
+                                        C.c_void_p, C.c_void_p]),
 }
 
 _lib: Optional[C.CDLL] = None
@@ -428,6 +430,15 @@ def q8_last_launch_info() -> dict:
     a, b, c, d, e = C.c_int(0), C.c_int(0), C.c_int(0), C.c_int(0), C.c_int(0)
     load().q8_last_launch_info(C.byref(a), C.byref(b), C.byref(c), C.byref(d), C.byref(e))
     return dict(gemm_kernel=a.value, launches=b.value, block_n=c.value, grid=d.value, ctas=e.value)
+
+
+def q8_measure_int8_mma_peak(ctas: int = 2, seconds: float = 0.2, dev_status=None, stream=None) -> dict:
+    """Issue-bound Int8 tensor-core rate of the current device (operands resident in shared memory)."""
+    tops, ms, sms = C.c_double(0.0), C.c_double(0.0), C.c_int(0)
+    st = load().q8_measure_int8_mma_peak(int(ctas), float(seconds), C.byref(tops), C.byref(ms), C.byref(sms),
+                                         _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
+    _check(st, "q8_measure_int8_mma_peak")
+    return dict(tops=tops.value, elapsed_ms=ms.value, sms_used=sms.value, ctas=int(ctas))
 
 
 def q8_tune_gemm_tail_split(enable: bool = True) -> None:
