@@ -223,6 +223,11 @@ void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *gri
  * SMs per 256 x 256 tile).  Results do not depend on the choice.  Not thread-safe. */
 q8_status q8_tune_gemm_tile(int block_n, int ctas);
 
+/* Tuning / test hook: epilogue warps per CTA of the cta_group::2 kernel for later calls in this process:
+ * 8 (each warp pipelines four 32-column blocks per tile through two staging buffers), 16 (two blocks per
+ * warp, one staging buffer) or 0 = automatic.  Other values are Q8_ERR_ARG.  Results do not depend on it. */
+q8_status q8_tune_gemm_epilogue_warps(int warps);
+
 /* Tuning / test hook for the schedule of the cta_group::2 kernel.  When the number of 256 x 256 tiles
  * is not a multiple of the number of SM pairs, the tiles of the last, partial round are cut into 2 or 4
  * narrower tiles (256 x 128 or 256 x 64) if these still fit in one round, which shortens that round.

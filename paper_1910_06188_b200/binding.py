@@ -50,6 +50,7 @@ SIGNATURES = {
     "q8_last_launch_info": (None, [C.POINTER(_int)] * 5),
     "q8_tune_gemm_tile": (_int, [_int, _int]),
     "q8_tune_gemm_tail_split": (None, [_int]),
+    "q8_tune_gemm_epilogue_warps": (_int, [_int]),
     "q8_last_launch_tail_split": (_int, []),
     "q8_measure_int8_mma_peak": (_int, [_int, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_int),
                                         C.c_void_p, C.c_void_p]),
@@ -439,6 +440,11 @@ def q8_measure_int8_mma_peak(ctas: int = 2, seconds: float = 0.2, dev_status=Non
                                          _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "q8_measure_int8_mma_peak")
     return dict(tops=tops.value, elapsed_ms=ms.value, sms_used=sms.value, ctas=int(ctas))
+
+
+def q8_tune_gemm_epilogue_warps(warps: int = 0) -> None:
+    """Forces 8 or 16 epilogue warps in the CTA-pair GEMM kernel for later calls (0 = automatic)."""
+    _check(load().q8_tune_gemm_epilogue_warps(int(warps)), "q8_tune_gemm_epilogue_warps")
 
 
 def q8_tune_gemm_tail_split(enable: bool = True) -> None:

@@ -446,6 +446,13 @@ q8_status q8_tune_gemm_tile(int block_n, int ctas)
     return Q8_OK;
 }
 
+q8_status q8_tune_gemm_epilogue_warps(int warps)
+{
+    if (warps != 0 && warps != 8 && warps != 16) return Q8_ERR_ARG;
+    set_gemm_epilogue_warps(warps);
+    return Q8_OK;
+}
+
 void q8_tune_gemm_tail_split(int enable) { set_gemm_tail_split(enable != 0); }
 
 int q8_last_launch_tail_split(void) { return last_launch_info().tail_split; }

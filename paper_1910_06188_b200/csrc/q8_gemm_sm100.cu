@@ -69,23 +69,31 @@ struct Cfg {
                                            | ((uint32_t)((BLOCK_M * CTAS) >> 4) << 24); // M / 16
 };
 
-// ---- GELU without erff: gelu(y) = max(y, 0) - a * Phi(-a), a = |y|, with
+// ---- GELU without erff, two values at a time: gelu(y) = max(y, 0) - a * Phi(-a), a = |y|, with
 // Phi(-a) = 2^p(a) and p a degree-6 fit of log2 Phi(-a) on [0, 5.6] (p(0) = -1 exactly; beyond 5.6
 // a * Phi(-a) < 1e-7 and a is clamped).  Absolute error of a * Phi(-a) below 1e-7, so the result is
-// within fp32 rounding of the erf form.  Six FMAs and one ex2 per element.
-__device__ __forceinline__ float gelu_fast(float y)
+// within fp32 rounding of the erf form.  The polynomial runs on packed fp32 FMAs (two values per
+// instruction, each half rounded like a scalar fmaf) in n = -a = max(-|y|, -5.6), i.e. with the odd
+// coefficients negated, so the last step needs no negation: gelu = n * 2^p + max(y, 0).
+// Per value: three packed FMA-pipe instructions and a half, one ex2, two min/max.
+__device__ __forceinline__ void gelu_fast_x2(uint64_t y2, float &out_lo, float &out_hi)
 {
-    const float a = fminf(fabsf(y), 5.6f);
-    float p = 2.9923698093625717e-05f;
-    p = fmaf(p, a, -0.0007398707093670964f);
-    p = fmaf(p, a, 0.007977453991770744f);
-    p = fmaf(p, a, -0.05323817580938339f);
-    p = fmaf(p, a, -0.45891568064689636f);
-    p = fmaf(p, a, -1.1511471271514893f);
-    p = fmaf(p, a, -1.0f);
-    float e;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(p));
-    return fmaf(-a, e, fmaxf(y, 0.0f));
+    float y0, y1;
+    unpack_f32x2(y2, y0, y1);
+    const uint64_t n = pack_f32x2(fmaxf(-fabsf(y0), -5.6f), fmaxf(-fabsf(y1), -5.6f));
+    uint64_t p = pack_f32x2(2.9923698093625717e-05f, 2.9923698093625717e-05f);
+    p = fma_f32x2(p, n, pack_f32x2(0.0007398707093670964f, 0.0007398707093670964f));
+    p = fma_f32x2(p, n, pack_f32x2(0.007977453991770744f, 0.007977453991770744f));
+    p = fma_f32x2(p, n, pack_f32x2(0.05323817580938339f, 0.05323817580938339f));
+    p = fma_f32x2(p, n, pack_f32x2(-0.45891568064689636f, -0.45891568064689636f));
+    p = fma_f32x2(p, n, pack_f32x2(1.1511471271514893f, 1.1511471271514893f));
+    p = fma_f32x2(p, n, pack_f32x2(-1.0f, -1.0f));
+    float p0, p1, e0, e1;
+    unpack_f32x2(p, p0, p1);
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(p0));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(p1));
+    const uint64_t r = fma_f32x2(n, pack_f32x2(e0, e1), pack_f32x2(fmaxf(y0, 0.0f), fmaxf(y1, 0.0f)));
+    unpack_f32x2(r, out_lo, out_hi);
 }
 
 // ------------------------------------------------------------------ epilogue of one warp
@@ -107,20 +115,16 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
     const bool row_ok = row < a.M;
     const float S_y = a.Yq != nullptr ? __ldg(a.S_y) : 1.0f;
     const bool yq_vec = ((a.N & 15) == 0) && ((reinterpret_cast<uintptr_t>(a.Yq) & 15u) == 0);
-#pragma unroll
-    for (int ci = 0; ci < NCHUNK; ++ci) {
-        if (ci >= nch) break;
+
+    // everything after the TMEM load, for the 32-column block ci held in v
+    auto finish_block = [&](uint32_t (&v)[32], int ci) {
         const int64_t nb = col0 + 32 * ci;
         const float inv = invv[ci];
+        if (nb >= a.N || row0 >= a.M) return;  // warp-uniform: the block lies outside the matrix
         // b_q of these 32 columns (one per lane, computed before the accumulator was ready) -> all lanes
         __syncwarp();
         bq_s[lane] = bqv[ci];
         __syncwarp();
-        uint32_t v[32];
-        tmem_ld_32x32(taddr + (uint32_t)(32 * ci), v);
-        tmem_ld_wait();
-        if (ci + 1 == nch) release();
-        if (nb >= a.N || row0 >= a.M) continue;  // warp-uniform: the block lies outside the matrix
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
             const int4 b = *reinterpret_cast<const int4 *>(bq_s + 4 * g);
@@ -136,9 +140,16 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
                 if (nb + j < a.N) drow[j] = (int32_t)v[j];
         }
         if (a.act == Q8_ACT_GELU) {
+            const uint64_t inv2 = pack_f32x2(inv, inv);
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-                v[j] = __float_as_uint(gelu_fast(__fmul_rn(__int2float_rn((int32_t)v[j]), inv)));
+            for (int j = 0; j < 32; j += 2) {
+                const uint64_t y2 =
+                    mul_f32x2(pack_f32x2(__int2float_rn((int32_t)v[j]), __int2float_rn((int32_t)v[j + 1])), inv2);
+                float g0, g1;
+                gelu_fast_x2(y2, g0, g1);
+                v[j] = __float_as_uint(g0);
+                v[j + 1] = __float_as_uint(g1);
+            }
         } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__fmul_rn(__int2float_rn((int32_t)v[j]), inv));
@@ -165,7 +176,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
                     if (nb + j < a.N) qrow[j] = (int8_t)quantize_value(__uint_as_float(v[j]), S_y);
             }
         }
-        if (a.Y == nullptr) continue;
+        if (a.Y == nullptr) return;
         if (tma_store) {
             if (lane == 0) tma_store_wait_read();  // the previous block has left the staging buffer
             __syncwarp();
@@ -183,6 +194,16 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
             for (int j = 0; j < 32; ++j)
                 if (nb + j < a.N) yrow[j] = __uint_as_float(v[j]);
         }
+    };
+
+#pragma unroll
+    for (int ci = 0; ci < NCHUNK; ++ci) {
+        if (ci >= nch) break;
+        uint32_t v[32];
+        tmem_ld_32x32(taddr + (uint32_t)(32 * ci), v);
+        tmem_ld_wait();
+        if (ci + 1 == nch) release();
+        finish_block(v, ci);
     }
 }
 
@@ -636,10 +657,11 @@ void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps)
 {
     g_force_block_n = block_n;
     g_force_ctas = ctas;
-    g_force_epilogue_warps = epilogue_warps;
+    if (epilogue_warps != 0) g_force_epilogue_warps = epilogue_warps;
 }
 
 void set_gemm_tail_split(bool enable) { g_tail_split_enabled = enable; }
+void set_gemm_epilogue_warps(int warps) { g_force_epilogue_warps = warps; }
 
 bool tcgen05_gemm_supported(const GemmArgs &a)
 {
