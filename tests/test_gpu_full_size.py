@@ -119,6 +119,39 @@ def test_split_tail_of_the_pair_schedule_matches_the_oracle(M, N, K, act):
         q8.q8_tune_gemm_tile(0, 0)
 
 
+@pytest.mark.parametrize("warps", [8, 16])
+def test_both_epilogue_widths_of_the_pair_kernel_match_the_oracle(warps):
+    from tests.gpu_util import check_linear
+    try:
+        q8.q8_tune_gemm_tile(256, 2)
+        q8.q8_tune_gemm_epilogue_warps(warps)
+        for (Mm, Nn, Kk, act) in [(700, 520, 272, 1), (515, 1030, 144, 0)]:
+            X = synth.activation(Mm, Kk, seed=1300 + Mm)
+            W = synth.weight(Nn, Kk, seed=1301 + Mm)
+            bb = synth.bias(Nn, seed=1302 + Mm)
+            info = check_linear(X, W, bb, act=act)
+            assert (info["block_n"], info["ctas"]) == (256, 2)
+    finally:
+        q8.q8_tune_gemm_epilogue_warps(0)
+        q8.q8_tune_gemm_tile(0, 0)
+    with pytest.raises(q8.Q8Error):
+        q8.q8_tune_gemm_epilogue_warps(12)
+
+
+def test_int8_mma_issue_peak_probe_runs_and_is_plausible():
+    """The measurement aid reports a rate between what the GEMM reaches and the datasheet's dense Int8 figure."""
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for ctas in (1, 2):
+        r = q8.q8_measure_int8_mma_peak(ctas, 0.01, dev_status=st)
+        assert st.item() == 0
+        assert r["sms_used"] == torch.cuda.get_device_properties(0).multi_processor_count // ctas * ctas
+        assert 1500.0 < r["tops"] < 6000.0, r
+    with pytest.raises(q8.Q8Error):
+        q8.q8_measure_int8_mma_peak(3, 0.01)
+    with pytest.raises(q8.Q8Error):
+        q8.q8_measure_int8_mma_peak(2, 100.0)
+
+
 def test_empty_problem_is_a_noop():
     Wq = torch.ones((8, 16), dtype=torch.int8, device="cuda")
     S = torch.ones(1, device="cuda")
