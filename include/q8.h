@@ -239,6 +239,16 @@ void q8_tune_gemm_tail_split(int enable);
  * of this host thread: 1 (not cut), 2 or 4. */
 int q8_last_launch_tail_split(void);
 
+/* q8_attention / q8_attention_quant run on the tensor cores when the padded sequence fits the accumulator
+ * memory (S rounded up to a multiple of 64, plus 64, at most 512 columns: S <= 448) and the pointers are
+ * 16-byte aligned: both products as tcgen05.mma kind::tf32 on operands split into a TF32-exact high part and a
+ * low remainder, three partial products accumulated in fp32, which keeps fp32-grade accuracy.  Otherwise, or
+ * after q8_tune_attention(0), a CUDA-core fp32 kernel computes the same thing.  The tensor-core kernel bounds
+ * its waits; a time-out sets the Q8_ERR_TIMEOUT bit in a per-device status word whose device address
+ * q8_attention_status_word returns (poll it with q8_poll_status).  Not thread-safe. */
+void q8_tune_attention(int use_tensor_cores);
+q8_status q8_attention_status_word(void **dev_status);
+
 /* Measurement aid, no counterpart in the paper: the issue-bound Int8 rate of the tensor cores of the current
  * device, i.e. the ceiling of the GEMM's tensor pipe when operands cost nothing.  Every SM (ctas = 1) or SM
  * pair (ctas = 2, cta_group::2) issues the GEMM kernel's own tcgen05.mma kind::i8 shape (M = 128 * ctas,

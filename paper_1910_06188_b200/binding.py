@@ -50,6 +50,8 @@ SIGNATURES = {
     "q8_last_launch_info": (None, [C.POINTER(_int)] * 5),
     "q8_tune_gemm_tile": (_int, [_int, _int]),
     "q8_tune_gemm_tail_split": (None, [_int]),
+    "q8_tune_attention": (None, [_int]),
+    "q8_attention_status_word": (_int, [C.POINTER(C.c_void_p)]),
     "q8_tune_gemm_epilogue_warps": (_int, [_int]),
     "q8_last_launch_tail_split": (_int, []),
     "q8_measure_int8_mma_peak": (_int, [_int, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_int),
@@ -440,6 +442,25 @@ def q8_measure_int8_mma_peak(ctas: int = 2, seconds: float = 0.2, dev_status=Non
                                          _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "q8_measure_int8_mma_peak")
     return dict(tops=tops.value, elapsed_ms=ms.value, sms_used=sms.value, ctas=int(ctas))
+
+
+def q8_tune_attention(use_tensor_cores: bool = True) -> None:
+    """Chooses between the tensor-core (3 x TF32) and the CUDA-core fp32 attention kernel for later calls."""
+    load().q8_tune_attention(1 if use_tensor_cores else 0)
+
+
+def q8_attention_status_word() -> int:
+    """Device address of the status word of the tensor-core attention kernel on the current device."""
+    p = C.c_void_p(0)
+    _check(load().q8_attention_status_word(C.byref(p)), "q8_attention_status_word")
+    return int(p.value)
+
+
+def q8_attention_status() -> Tuple[int, int]:
+    """Synchronises, reads and clears the status word of the tensor-core attention kernel."""
+    raw = C.c_uint32(0)
+    st = load().q8_poll_status(C.c_void_p(q8_attention_status_word()), C.byref(raw), None)
+    return int(st), int(raw.value)
 
 
 def q8_tune_gemm_epilogue_warps(warps: int = 0) -> None:

@@ -453,6 +453,15 @@ q8_status q8_tune_gemm_epilogue_warps(int warps)
     return Q8_OK;
 }
 
+void q8_tune_attention(int use_tensor_cores) { set_attention_tensor_cores(use_tensor_cores != 0); }
+
+q8_status q8_attention_status_word(void **dev_status)
+{
+    if (dev_status == nullptr) return Q8_ERR_NULL;
+    *dev_status = attention_status_word();
+    return *dev_status != nullptr ? Q8_OK : Q8_ERR_CUDA;
+}
+
 void q8_tune_gemm_tail_split(int enable) { set_gemm_tail_split(enable != 0); }
 
 int q8_last_launch_tail_split(void) { return last_launch_info().tail_split; }

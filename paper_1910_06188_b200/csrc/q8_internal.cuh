@@ -72,6 +72,13 @@ cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r
 cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
                              int8_t *ctx_q, cudaStream_t s);
 
+// Tensor-core attention (q8_attention_sm100.cu): 3 x TF32 split products with fp32 accumulation in TMEM.
+bool attention_tc_supported(const float *qkv, int64_t S, int64_t heads, const float *ctx, const int8_t *ctx_q);
+cudaError_t launch_attention_tc(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
+                                int8_t *ctx_q, cudaStream_t s);
+void set_attention_tensor_cores(bool enable);
+int32_t *attention_status_word();  // device word that receives Q8_ERR_TIMEOUT from the tensor-core attention kernel
+
 // ---- GEMM launchers ----
 bool tcgen05_gemm_supported(const GemmArgs &a);
 void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps = 0);  // 0, 0 = automatic choice

@@ -364,6 +364,7 @@ cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t hea
                              int8_t *ctx_q, cudaStream_t s)
 {
     if (B <= 0 || S <= 0 || heads <= 0) return cudaSuccess;
+    if (attention_tc_supported(qkv, S, heads, ctx, ctx_q)) return launch_attention_tc(qkv, B, S, heads, ctx, S_q, ctx_q, s);
     static bool attr_set[64] = {};  // opt-in shared-memory size: per device, per function
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);

@@ -43,6 +43,22 @@ def test_attention(B, S, heads):
     assert_close_fp(got, o.attention(qkv, B, S, heads), "attention")
 
 
+@pytest.mark.parametrize("B,S,heads", [(2, 100, 2), (1, 384, 2), (1, 448, 1), (1, 500, 1)])
+def test_attention_tensor_core_and_cuda_core_kernels_both_match_the_oracle(B, S, heads):
+    """S <= 448 runs on the tensor cores (split TF32 products), longer sequences and q8_tune_attention(0)
+    on the CUDA-core kernel; both must meet the fp32 tolerance."""
+    qkv = synth.normal((B * S, 3 * heads * 64), 1.0, 3150 + S)
+    ref = o.attention(qkv, B, S, heads)
+    try:
+        for tensor_cores in (True, False):
+            q8.q8_tune_attention(tensor_cores)
+            got = q8.q8_attention(dev(qkv), B, S, heads).cpu().numpy()
+            assert q8.q8_attention_status() == (q8.Q8_OK, 0)
+            assert_close_fp(got, ref, f"attention (tensor cores {tensor_cores})")
+    finally:
+        q8.q8_tune_attention(True)
+
+
 def test_attention_large_logits_stay_finite():
     B, S, heads = 1, 130, 1
     qkv = synth.normal((B * S, 3 * 64), 6.0, 3150)             # logits of several hundred
