@@ -539,7 +539,7 @@ def run_ours(args):
 
 
 def measure_small_cases(args, torch, q8):
-    """The two smaller BASELINE configurations, timed as back-to-back calls (their data fits in L2, so these are
+    """The two smaller workload configurations, timed as back-to-back calls (their data fits in L2, so these are
     L2-warm, launch-latency-dominated figures; reported in microseconds rather than against a roofline)."""
     out = {}
     dev = torch.device("cuda", torch.cuda.current_device())

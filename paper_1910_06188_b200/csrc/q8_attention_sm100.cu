@@ -10,9 +10,9 @@
 // All operands are staged by the workers themselves (global -> registers -> split -> shared memory in the
 // K-major 128-byte-swizzled layout the MMA reads); no TMA, no multicast.  Chunks of 64 keys go through two
 // buffer sets, so the MMAs of chunk c run while the workers prepare chunk c + 1:
-//   phase 1  Q tile (scaled by log2(e)/8) -> Q_hi, Q_lo; per chunk: K chunk -> K_hi, K_lo; 24 MMAs (2 swizzle
-//            spans x 4 K steps x 3 partial products) -> scores in TMEM columns [64 c, 64 c + 64); the row maxima
-//            are read from TMEM chunk by chunk behind the MMAs (a row is shared by four threads)
+//   phase 1  Q tile (scaled by log2(e)/8) -> Q_hi, Q_lo; per 128 keys: K rows -> K_hi, K_lo; 24 MMAs with N = 128
+//            (2 swizzle spans x 4 K steps x 3 partial products) -> scores in TMEM columns [128 c, 128 c + 128); the
+//            row maxima are read from TMEM chunk by chunk behind the MMAs (a row is shared by four threads)
 //   phase 2  per chunk: p = 2^(s - max) -> P_hi, P_lo (A operand, keys along K); V chunk transposed ->
 //            [V_hi ; V_lo] stacked as one 128-row B operand, so that one N = 128 MMA yields P_hi V_hi (columns
 //            0..63 of the O accumulator) and P_hi V_lo (columns 64..127), and one N = 64 MMA adds P_lo V_hi to the
@@ -43,6 +43,13 @@ constexpr int kLoRowsB = kChunk * 128;         // offset of the lo rows inside a
 constexpr int kBufQP = 4 * kSpanBytesA;        // {hi, lo} x 2 spans: Q, then P
 constexpr int kBufKV = 2 * kSpanBytesB;        // 2 spans x [hi ; lo]: K, then V^T
 constexpr int kAttnTcSmemBytes = 1024 + 2 * kBufQP + 2 * kBufKV;  // two buffer sets: 193 KB
+// Phase 1 takes keys 128 at a time (N = 128 score MMAs: half as many instructions, each reading Q once for twice
+// the columns).  Its two K buffers of 64 KB ([hi 128 rows | lo 128 rows] per span) lie over the four phase-2
+// buffers behind Q.
+constexpr int kBigChunk = 2 * kChunk;
+constexpr int kSpanBytesK = 2 * kBigChunk * 128;  // one span of a 128-key K buffer, hi rows then lo rows: 32 KB
+constexpr int kLoRowsK = kBigChunk * 128;
+static_assert(2 * (2 * kSpanBytesK) == 2 * kBufKV + kBufQP, "the two K buffers of phase 1 cover K/V 0, K/V 1 and P 1");
 
 // tcgen05.mma kind::tf32 instruction descriptor: D = F32, A = B = TF32, both K-major, M = 128.
 constexpr uint32_t kIdescBase = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kQTile >> 4) << 24);
@@ -88,6 +95,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
     // [ Q, then P buffer 0 | K / V buffer 0 | K / V buffer 1 | P buffer 1 ]
     uint8_t *const q_buf = smem;
     auto kv_buf = [&](int b) { return smem + kBufQP + b * kBufKV; };
+    auto k_buf = [&](int b) { return smem + kBufQP + b * (2 * kSpanBytesK); };  // phase 1 only
     auto p_buf = [&](int b) { return smem + b * (kBufQP + 2 * kBufKV); };
     __shared__ __align__(8) uint64_t ready_bar[2];  // workers -> MMA warp: the operands of a chunk are in place
     __shared__ __align__(8) uint64_t done_bar[2];   // MMA warp -> workers: the MMAs of a chunk have completed
@@ -102,6 +110,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
     const float *base = qkv + seq * (int64_t)S * row_pitch + head * kHeadDim;
     const int chunks = (S + kChunk - 1) / kChunk;
     const int s_pad = chunks * kChunk;
+    const int big_chunks = (S + kBigChunk - 1) / kBigChunk;
 
     if (tid == 0) {
         for (int b = 0; b < 2; ++b) {
@@ -124,24 +133,24 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             uint32_t ready_phase = 0u;  // bit b: parity of the next phase of ready_bar[b]
             bool ok = true;
             const uint32_t q_hi = smem_u32(q_buf), q_lo = q_hi + 2 * kSpanBytesA;
-            for (int kc = 0; kc < chunks && ok; ++kc) {  // scores of chunk kc
+            for (int kc = 0; kc < big_chunks && ok; ++kc) {  // scores of the 128 keys of big chunk kc
                 const int b = kc & 1;
                 ok = mbar_wait(smem_u32(&ready_bar[b]), (ready_phase >> b) & 1u, &abort_flag, status);
                 ready_phase ^= 1u << b;
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d = tmem_base + (uint32_t)(kc * kChunk), kb = smem_u32(kv_buf(b));
+                const uint32_t d = tmem_base + (uint32_t)(kc * kBigChunk), kb = smem_u32(k_buf(b));
                 uint32_t acc = 0u;
 #pragma unroll
                 for (int span = 0; span < 2; ++span) {
                     const uint64_t ah = smem_desc_sw128(q_hi + span * kSpanBytesA), al = smem_desc_sw128(q_lo + span * kSpanBytesA);
-                    const uint64_t bh = smem_desc_sw128(kb + span * kSpanBytesB), bl = smem_desc_sw128(kb + span * kSpanBytesB + kLoRowsB);
+                    const uint64_t bh = smem_desc_sw128(kb + span * kSpanBytesK), bl = smem_desc_sw128(kb + span * kSpanBytesK + kLoRowsK);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {  // 8 fp32 = 32 bytes of K per instruction: +2 in the (address >> 4) field
                         const uint64_t adv = (uint64_t)(2 * ks);
-                        umma_tf32(d, al + adv, bh + adv, kIdescN64, acc);  // small terms first
-                        umma_tf32(d, ah + adv, bl + adv, kIdescN64, 1u);
-                        umma_tf32(d, ah + adv, bh + adv, kIdescN64, 1u);
+                        umma_tf32(d, al + adv, bh + adv, kIdescN128, acc);  // small terms first
+                        umma_tf32(d, ah + adv, bl + adv, kIdescN128, 1u);
+                        umma_tf32(d, ah + adv, bh + adv, kIdescN128, 1u);
                         acc = 1u;
                     }
                 }
@@ -204,9 +213,9 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             uint8_t *at = q_buf + (pc >> 3) * kSpanBytesA + sw128_offset(r, pc & 7);
             store_split4(at, at + 2 * kSpanBytesA, v);
         }
-        constexpr int kPiecesK = (kChunk * 16) / kWorkers;  // 16-byte pieces of a K chunk per thread
+        constexpr int kPiecesK = (kBigChunk * 16) / kWorkers;  // 16-byte pieces of a 128-key K chunk per thread
         float4 kreg[kPiecesK];
-        auto fetch_k = [&](int j0) {  // 64 keys x 64 fp32
+        auto fetch_k = [&](int j0) {  // 128 keys x 64 fp32
 #pragma unroll
             for (int i = 0; i < kPiecesK; ++i) {
                 const int c = tid + i * kWorkers, r = c >> 4, pc = c & 15;
@@ -215,24 +224,24 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             }
         };
         float m = -INFINITY;
-        auto take_max = [&](int c) {  // this thread's 16 columns of chunk c
-            uint32_t v[16];
-            const int col0 = c * kChunk + cq * 16;
-            tmem_ld_32x16(t_row + (uint32_t)col0, v);
+        auto take_max = [&](int c) {  // this thread's 32 columns of big chunk c
+            uint32_t v[32];
+            const int col0 = c * kBigChunk + cq * 32;
+            tmem_ld_32x32(t_row + (uint32_t)col0, v);
             tmem_ld_wait();
-            if (col0 + 16 <= S) {
+            if (col0 + 32 <= S) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) m = fmaxf(m, __uint_as_float(v[j]));
+                for (int j = 0; j < 32; ++j) m = fmaxf(m, __uint_as_float(v[j]));
             } else {
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
+                for (int j = 0; j < 32; ++j)
                     if (col0 + j < S) m = fmaxf(m, __uint_as_float(v[j]));
             }
         };
         fetch_k(0);
-        for (int kc = 0; kc < chunks && ok; ++kc) {
+        for (int kc = 0; kc < big_chunks && ok; ++kc) {
             const int b = kc & 1;
-            if (kc >= 2) {  // buffer set b was read by the MMAs of chunk kc - 2, whose scores are final after this wait
+            if (kc >= 2) {  // buffer b was read by the MMAs of big chunk kc - 2, whose scores are final after this wait
                 wait_done(b);
                 if (!ok) break;
                 take_max(kc - 2);
@@ -240,13 +249,13 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
 #pragma unroll
             for (int i = 0; i < kPiecesK; ++i) {
                 const int c = tid + i * kWorkers, r = c >> 4, pc = c & 15;
-                uint8_t *at = kv_buf(b) + (pc >> 3) * kSpanBytesB + sw128_offset(r, pc & 7);
-                store_split4(at, at + kLoRowsB, kreg[i]);
+                uint8_t *at = k_buf(b) + (pc >> 3) * kSpanBytesK + sw128_offset(r, pc & 7);
+                store_split4(at, at + kLoRowsK, kreg[i]);
             }
-            if (kc + 1 < chunks) fetch_k((kc + 1) * kChunk);  // next K chunk, in flight during the MMAs
+            if (kc + 1 < big_chunks) fetch_k((kc + 1) * kBigChunk);  // next K chunk, in flight during the MMAs
             report_ready(b);
         }
-        for (int c = (chunks > 2 ? chunks - 2 : 0); c < chunks && ok; ++c) {  // the last two chunks
+        for (int c = (big_chunks > 2 ? big_chunks - 2 : 0); c < big_chunks && ok; ++c) {  // the last two big chunks
             wait_done(c & 1);
             if (ok) take_max(c);
         }
