@@ -261,6 +261,17 @@ q8_status q8_attention_status_word(void **dev_status);
 q8_status q8_measure_int8_mma_peak(int ctas, double seconds, double *tops, double *elapsed_ms, int *sms_used,
                                    void *dev_status, void *stream);
 
+/* Measurement aid, no counterpart in the paper: the one-directional HBM rates of the current device.  A copy
+ * moves one byte in per byte out; the FC layers write 4 M N bytes of fp32 against M K + N K bytes of Int8
+ * operands, so what bounds their output-heavy shapes is the store-only rate, which is well below the copy rate.
+ * `buf` (device, 16-byte aligned, caller-owned, at least `bytes` long; make it several times the L2 size) is
+ * overwritten with a pattern `repeats` times (store != 0) or read `repeats` times (store == 0) by a plain
+ * grid-stride kernel of 16-byte accesses after one untimed pass.  Host outputs: *gbs = bytes * repeats / time in
+ * 1e9 B/s (required), *elapsed_ms (may be NULL).  Synchronises `stream`.  Allocates no device memory.
+ * Returns Q8_ERR_NULL / Q8_ERR_ALIGN / Q8_ERR_ARG (bytes < 16, repeats outside 1..1000) / Q8_ERR_CUDA. */
+q8_status q8_measure_hbm_peak(void *buf, size_t bytes, int store, int repeats, double *gbs, double *elapsed_ms,
+                              void *stream);
+
 #ifdef __cplusplus
 }
 #endif

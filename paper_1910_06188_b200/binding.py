@@ -54,6 +54,8 @@ SIGNATURES = {
     "q8_attention_status_word": (_int, [C.POINTER(C.c_void_p)]),
     "q8_tune_gemm_epilogue_warps": (_int, [_int]),
     "q8_last_launch_tail_split": (_int, []),
+    "q8_measure_hbm_peak": (_int, [C.c_void_p, C.c_size_t, _int, _int, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                   C.c_void_p]),
     "q8_measure_int8_mma_peak": (_int, [_int, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_int),
                                         C.c_void_p, C.c_void_p]),
 }
@@ -442,6 +444,16 @@ def q8_measure_int8_mma_peak(ctas: int = 2, seconds: float = 0.2, dev_status=Non
                                          _ptr(dev_status, torch.int32, "dev_status"), _stream(stream))
     _check(st, "q8_measure_int8_mma_peak")
     return dict(tops=tops.value, elapsed_ms=ms.value, sms_used=sms.value, ctas=int(ctas))
+
+
+def q8_measure_hbm_peak(buf: torch.Tensor, store: bool, repeats: int = 10, stream=None) -> dict:
+    """Store-only (or load-only) HBM rate over the caller's device buffer `buf`, in GB/s."""
+    gbs, ms = C.c_double(0.0), C.c_double(0.0)
+    nbytes = buf.numel() * buf.element_size()
+    st = load().q8_measure_hbm_peak(_any_ptr(buf, "buf"), nbytes, 1 if store else 0, int(repeats), C.byref(gbs),
+                                    C.byref(ms), _stream(stream))
+    _check(st, "q8_measure_hbm_peak")
+    return {"gbs": gbs.value, "elapsed_ms": ms.value, "bytes": nbytes, "repeats": int(repeats), "store": bool(store)}
 
 
 def q8_tune_attention(use_tensor_cores: bool = True) -> None:

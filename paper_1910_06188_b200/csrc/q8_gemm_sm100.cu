@@ -106,15 +106,22 @@ __device__ __forceinline__ void gelu_fast_x2(uint64_t y2, float &out_lo, float &
 // Once the last TMEM load of the tile has landed the accumulator buffer is handed back (release()).
 template <int COLS, typename Release>
 __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
-                                              uint32_t taddr, int64_t row0, int64_t col0, const int32_t (&bqv)[COLS / 32],
-                                              const float (&invv)[COLS / 32], uint8_t *stage, int32_t *bq_s, int lane, int nch,
-                                              Release release)
+                                              const CUtensorMap *tmap_yq, bool yq_tma, uint32_t taddr, int64_t row0,
+                                              int64_t col0, const int32_t (&bqv)[COLS / 32], const float (&invv)[COLS / 32],
+                                              uint8_t *stage, int32_t *bq_s, int lane, int nch, Release release)
 {
     constexpr int NCHUNK = COLS / 32;  // compile-time maximum; this tile has nch <= NCHUNK blocks (warp-uniform)
     const int64_t row = row0 + lane;
     const bool row_ok = row < a.M;
     const float S_y = a.Yq != nullptr ? __ldg(a.S_y) : 1.0f;
     const bool yq_vec = ((a.N & 15) == 0) && ((reinterpret_cast<uintptr_t>(a.Yq) & 15u) == 0);
+    // Int8-only output of a full-width tile: the warp's 32 x COLS bytes are collected in its staging buffer (free,
+    // since no fp32 block is staged) in the swizzled layout of the Int8 output tensor map and leave as one TMA
+    // store of whole 64- or 128-byte row pieces instead of 32 separate 16-byte stores per lane and block.
+    constexpr bool kYqStageable = COLS == 64 || COLS == 128;
+    const bool yq_staged = kYqStageable && yq_tma && nch == NCHUNK;
+    const int yq_xor = COLS == 128 ? (lane & 7) : ((lane >> 1) & 3);  // 128-byte / 64-byte swizzle of row `lane`
+    bool yq_pending = false;
 
     // everything after the TMEM load, for the 32-column block ci held in v
     auto finish_block = [&](uint32_t (&v)[32], int ci) {
@@ -157,7 +164,9 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
         if (a.Yq != nullptr && row_ok) {
             // re-quantised output for the next quantised layer: Eq. 1 at that layer's activation scale
             int8_t *qrow = a.Yq + row * a.N + nb;
-            if (yq_vec) {  // N % 16 == 0: a 16-byte piece is never split by the edge
+            if (yq_staged) {
+                // handled below, for all rows of the warp (rows past M are clipped by the store)
+            } else if (yq_vec) {  // N % 16 == 0: a 16-byte piece is never split by the edge
                 if (nb < a.N)
                     *reinterpret_cast<uint4 *>(qrow) = make_uint4(
                         quantize_pack4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]), S_y),
@@ -175,6 +184,24 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
                 for (int j = 0; j < 32; ++j)
                     if (nb + j < a.N) qrow[j] = (int8_t)quantize_value(__uint_as_float(v[j]), S_y);
             }
+        }
+        if (yq_staged) {
+            if (!yq_pending) {
+                if (lane == 0) tma_store_wait_read();  // the previous tile has left the staging buffer
+                __syncwarp();
+                yq_pending = true;
+            }
+            uint8_t *srow = stage + lane * COLS;
+            *reinterpret_cast<uint4 *>(srow + (((2 * ci) ^ yq_xor) << 4)) = make_uint4(
+                quantize_pack4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]), S_y),
+                quantize_pack4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]), S_y),
+                quantize_pack4(__uint_as_float(v[8]), __uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]), S_y),
+                quantize_pack4(__uint_as_float(v[12]), __uint_as_float(v[13]), __uint_as_float(v[14]), __uint_as_float(v[15]), S_y));
+            *reinterpret_cast<uint4 *>(srow + (((2 * ci + 1) ^ yq_xor) << 4)) = make_uint4(
+                quantize_pack4(__uint_as_float(v[16]), __uint_as_float(v[17]), __uint_as_float(v[18]), __uint_as_float(v[19]), S_y),
+                quantize_pack4(__uint_as_float(v[20]), __uint_as_float(v[21]), __uint_as_float(v[22]), __uint_as_float(v[23]), S_y),
+                quantize_pack4(__uint_as_float(v[24]), __uint_as_float(v[25]), __uint_as_float(v[26]), __uint_as_float(v[27]), S_y),
+                quantize_pack4(__uint_as_float(v[28]), __uint_as_float(v[29]), __uint_as_float(v[30]), __uint_as_float(v[31]), S_y));
         }
         if (a.Y == nullptr) return;
         if (tma_store) {
@@ -205,6 +232,12 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
         if (ci + 1 == nch) release();
         finish_block(v, ci);
     }
+    if (yq_pending) {
+        // blocks beyond column N were never staged; the store clips them (and rows past M) at the matrix edge
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) tma_store_2d(tmap_yq, (int32_t)col0, (int32_t)row0, smem_u32(stage));
+    }
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -212,7 +245,8 @@ template <int BLOCK_N, int CTAS, int EW>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_w4,
-                    const __grid_constant__ CUtensorMap tmap_y, GemmArgs a, int tma_store, int64_t full_tiles, int split)
+                    const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_yq, GemmArgs a,
+                    int tma_store, int yq_tma, int64_t full_tiles, int split)
 {
     using C = Cfg<BLOCK_N, CTAS, EW>;
     constexpr int kEpilogueWarps = EW;
@@ -450,7 +484,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
             };
             if (active)
-                epilogue_warp<C::kColsPerWarp>(a, &tmap_y, tma_store != 0,
+                epilogue_warp<C::kColsPerWarp>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                                                m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release);
             else
@@ -522,6 +556,22 @@ bool make_tmap_out(CUtensorMap *map, float *base, int64_t M, int64_t N)
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// Row-major Int8 output [M, N] as a tensor map of (box_cols x 32) boxes: 64-byte rows with the 64-byte swizzle
+// or 128-byte rows with the 128-byte swizzle.
+bool make_tmap_out_q(CUtensorMap *map, int8_t *base, int64_t M, int64_t N, int box_cols)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    cuuint64_t strides[1] = {(cuuint64_t)N};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    box_cols == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -604,6 +654,12 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     } else {
         ty = tx;  // never dereferenced
     }
+    // Int8-only output (no fp32 Y): full-width tiles leave through TMA stores of the staged Int8 rows
+    CUtensorMap tyq = tx;  // never dereferenced unless yq_tma
+    constexpr int kCpw = C::kColsPerWarp;
+    int yq_tma = (kCpw == 64 || kCpw == 128) && a.Y == nullptr && a.Yq != nullptr && ((a.N & 15) == 0) &&
+                 ((reinterpret_cast<uintptr_t>(a.Yq) & 15u) == 0);
+    if (yq_tma && !make_tmap_out_q(&tyq, a.Yq, a.M, a.N, kCpw)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(units * CTAS));
     cfg.blockDim = dim3(kThreads);
@@ -616,7 +672,7 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, kernel, tx, tw, tw2, tw4, ty, a, tma_store, full_tiles, split);
+    e = cudaLaunchKernelEx(&cfg, kernel, tx, tw, tw2, tw4, ty, tyq, a, tma_store, yq_tma, full_tiles, split);
     LaunchInfo &li = last_launch_info();
     li.gemm_kernel = 1;
     li.block_n = BLOCK_N;

@@ -138,6 +138,49 @@ def test_both_epilogue_widths_of_the_pair_kernel_match_the_oracle(warps):
         q8.q8_tune_gemm_epilogue_warps(12)
 
 
+@pytest.mark.parametrize("block_n,ctas,warps", [(32, 1, 0), (64, 1, 0), (128, 1, 0), (256, 1, 0), (256, 2, 8), (256, 2, 16)])
+def test_int8_only_output_of_every_tile_shape(block_n, ctas, warps):
+    """The Int8-only output (no fp32 Y; what FFN1 hands to FFN2) leaves full-width tiles through staged TMA
+    stores and narrow or ragged ones lane by lane: either way it must be Eq. 1 applied to exactly the fp32
+    value the plain call stores, and nothing may be written outside the matrix."""
+    shapes = [(515, 1040, 272, 1), (700, 528, 144, 0), (100, 16, 64, 1)]
+    if ctas == 2:
+        shapes.append((20000, 1008, 128, 1))  # partial last round: tail tiles cut into narrower ones
+    S_y = dev(np.array([23.0], np.float32))
+    try:
+        q8.q8_tune_gemm_tile(block_n, ctas)
+        q8.q8_tune_gemm_epilogue_warps(warps)
+        for (Mm, Nn, Kk, act) in shapes:
+            Xq = dev((synth.token_ids(Mm * Kk, 255, seed=1600 + Mm) - 127).astype(np.int8).reshape(Mm, Kk))
+            Wq, S_w = q8.q8_quantize_weight(dev(synth.weight(Nn, Kk, seed=1601 + Mm)))
+            bb = dev(synth.bias(Nn, seed=1602 + Mm))
+            S_x = dev(np.array([6.0], np.float32))
+            Y = q8.q8_linear_q(Xq, S_x, Wq, S_w, bb, act)
+            assert (q8.q8_last_launch_info()["block_n"], q8.q8_last_launch_info()["ctas"]) == (block_n, ctas)
+            buf = torch.full((Mm * Nn + 256,), 77, dtype=torch.int8, device="cuda")
+            Yq = buf[128: 128 + Mm * Nn].view(Mm, Nn)
+            st = torch.zeros(1, dtype=torch.int32, device="cuda")
+            q8.q8_linear_q_requant(Xq, S_x, Wq, S_w, bb, act, S_y, Yq=Yq, dev_status=st)
+            assert q8.q8_poll_status(st) == (q8.Q8_OK, 0)
+            assert np.array_equal(Yq.cpu().numpy(), o.quantize(Y.cpu().numpy(), 23.0)), (Mm, Nn, Kk)
+            assert torch.all(buf[:128] == 77) and torch.all(buf[128 + Mm * Nn:] == 77)
+    finally:
+        q8.q8_tune_gemm_epilogue_warps(0)
+        q8.q8_tune_gemm_tile(0, 0)
+
+
+def test_hbm_peak_probe_runs_and_is_plausible():
+    buf = torch.empty(1 << 29, dtype=torch.uint8, device="cuda")
+    w = q8.q8_measure_hbm_peak(buf, store=True, repeats=5)
+    r = q8.q8_measure_hbm_peak(buf, store=False, repeats=5)
+    assert 500.0 < w["gbs"] < 12000.0 and 500.0 < r["gbs"] < 12000.0
+    assert buf[:16].cpu().numpy().tolist() != [0] * 16  # the store pass did write
+    with pytest.raises(q8.Q8Error):
+        q8.q8_measure_hbm_peak(buf[1:], store=True)  # misaligned
+    with pytest.raises(q8.Q8Error):
+        q8.q8_measure_hbm_peak(buf, store=True, repeats=0)
+
+
 def test_int8_mma_issue_peak_probe_runs_and_is_plausible():
     """The measurement aid reports a rate between what the GEMM reaches and the datasheet's dense Int8 figure."""
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
