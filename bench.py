@@ -40,9 +40,10 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of the tcgen05 GEMM per launch on the BERT-Large FC set, from the
 # ncu captures summarised in profiles/gemm_tcgen05_dram_traffic_m24576.md (one layer resident per capture).  Below the
 # algorithmic bytes because part of each output is still dirty in the 126 MB L2 when the kernel ends.
-GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 270164992, "attn_out": 67688192, "ffn1": 372135680, "ffn2": 164227584}}
+GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 269510144, "attn_out": 67068928, "ffn1": 371191040, "ffn2": 163424768}}
 NOMINAL_INT8_OVER_BF16 = 2.0  # dense tensor peak ratio int8 : bf16 (4.5 : 2.25 POPS nominal)
 GEMM_REPS = 4  # launches per event pair in the per-kernel pass
+EMB_REPS = 4   # embedding gathers per event pair in the per-kernel pass
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -277,17 +278,46 @@ def run_ours(args):
         if code != q8.Q8_OK:
             raise SystemExit(f"device status {code} ({q8.status_string(code)}) on layer {L['name']}")
 
+    # One step is a fixed sequence of launches on fixed buffers, so it is captured once in a CUDA graph and the
+    # timed region replays that graph (no host work between the kernels); --no-graph times the eager launches.
+    step_graph = None
+    if not args.no_graph and not args.profile_mode and n_streams == 1:
+        try:
+            step_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(step_graph):
+                step()
+            for _ in range(3):
+                step_graph.replay()
+            barrier()
+        except Exception as ex:  # capture is an optimisation of the launch path only
+            print(f"[bench] CUDA graph capture failed ({ex}); timing eager launches", file=sys.stderr)
+            step_graph = None
+            step()
+            barrier()
+
     # ---- timed region: K whole steps, device time, max over ranks
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local_rank)
+    eager_ms = None
     with sampler:
         barrier()
         ev0.record(stream)
         for _ in range(args.steps):
-            step()
+            if step_graph is not None:
+                step_graph.replay()
+            else:
+                step()
         ev1.record(stream)
         barrier()
         ms = ev0.elapsed_time(ev1)
+        if step_graph is not None:
+            # the same K steps launched eagerly from the host, reported beside the graph-replayed figure
+            ev0.record(stream)
+            for _ in range(args.steps):
+                step()
+            ev1.record(stream)
+            barrier()
+            eager_ms = ev0.elapsed_time(ev1) / args.steps
 
         # ---- per-kernel pass (same launches, events around each kernel): roofline of the dominant kernel
         nl = len(layers)
@@ -302,22 +332,59 @@ def run_ours(args):
         for i, L in enumerate(layers):
             groups.setdefault(L["M"] * L["K"], []).append(i)
         gev = {k: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for k in groups}
+        # The launches between two events are replayed from a CUDA graph, so the events see device time without
+        # host gaps: each layer's GEMM_REPS back-to-back GEMM launches, each group of quantise passes, and
+        # EMB_REPS embedding gathers that alternate between two output buffers (together larger than L2).
+        gemm_graphs, quant_graphs, emb_graph = [], {}, None
+        emb_out2 = torch.empty_like(emb_out) if ksteps > 0 else None
+        if not args.no_graph and ksteps > 0:
+            try:
+                for L in layers:
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g):
+                        for _ in range(GEMM_REPS):
+                            q8.q8_linear_q(L["Xq"], L["S_x"], L["Wq"], L["S_w"], L["bd"], L["act"], Y=L["Y"])
+                    gemm_graphs.append(g)
+                for k, members in groups.items():
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g):
+                        for i in members:
+                            q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
+                    quant_graphs[k] = g
+                emb_graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(emb_graph):
+                    for r in range(EMB_REPS):
+                        q8.q8_embedding(ids, Eq, S_e, out=emb_out if r % 2 == 0 else emb_out2)
+                torch.cuda.synchronize()
+            except Exception as ex:
+                print(f"[bench] CUDA graph capture of the per-kernel pass failed ({ex}); timing eager launches", file=sys.stderr)
+                gemm_graphs, quant_graphs, emb_graph = [], {}, None
         for _ in range(ksteps):
             ev_e0.record(stream)
-            q8.q8_embedding(ids, Eq, S_e, out=emb_out)
+            if emb_graph is not None:
+                emb_graph.replay()
+            else:
+                for r in range(EMB_REPS):
+                    q8.q8_embedding(ids, Eq, S_e, out=emb_out if r % 2 == 0 else emb_out2)
             ev_e1.record(stream)
             for k, members in groups.items():
                 gev[k][0].record(stream)
-                for i in members:
-                    q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
+                if k in quant_graphs:
+                    quant_graphs[k].replay()
+                else:
+                    for i in members:
+                        q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
                 gev[k][1].record(stream)
             for i, L in enumerate(layers):
                 evs[i][1].record(stream)
-                for _ in range(GEMM_REPS):  # back to back, so that the event overhead is shared by several launches
-                    q8.q8_linear_q(L["Xq"], L["S_x"], L["Wq"], L["S_w"], L["bd"], L["act"], Y=L["Y"])
+                if gemm_graphs:
+                    gemm_graphs[i].replay()
+                else:
+                    for _ in range(GEMM_REPS):  # back to back, so that the event overhead is shared by several launches
+                        q8.q8_linear_q(L["Xq"], L["S_x"], L["Wq"], L["S_w"], L["bd"], L["act"], Y=L["Y"])
                 evs[i][2].record(stream)
             torch.cuda.synchronize()
-            t_emb += ev_e0.elapsed_time(ev_e1)
+            t_emb += ev_e0.elapsed_time(ev_e1) / EMB_REPS
             for k, members in groups.items():
                 for i in members:
                     t_quant[i] += gev[k][0].elapsed_time(gev[k][1]) / len(members)
@@ -453,6 +520,33 @@ def run_ours(args):
             "what": "tcgen05.mma cta_group::2 kind::i8 256x256x32 issued back to back on all SM pairs, operands resident "
                     "in shared memory, no loads or stores (q8_measure_int8_mma_peak)",
         }
+    # One-directional HBM rates measured now (a copy moves a byte in per byte out; the fp32 output of an FC layer
+    # is almost pure store traffic): the floor of a layer is the slower of its MMAs at the Int8 peak and its
+    # 4 M N output bytes at the store-only rate.
+    hbm_dir = None
+    if world == 1:
+        probe = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+        st_r = q8.q8_measure_hbm_peak(probe, store=True, repeats=10)
+        ld_r = q8.q8_measure_hbm_peak(probe, store=False, repeats=10)
+        del probe
+        t_floor = []
+        for L, go, bl in zip(layers, gemm_ops, by_layer):
+            y_bytes = 4.0 * L["M"] * L["N"]
+            t_tensor = go / (int8_peak * 1e12)
+            t_store = y_bytes / (st_r["gbs"] * 1e9)
+            t_floor.append(max(t_tensor, t_store))
+            bl["gemm_y_store_gbs"] = y_bytes / (bl["gemm_us"] * 1e-6) / 1e9
+            bl["gemm_frac_hbm_store"] = bl["gemm_y_store_gbs"] / st_r["gbs"]
+            bl["gemm_floor_us"] = t_floor[-1] * 1e6
+            bl["gemm_floor_bound"] = "hbm_store" if t_store > t_tensor else "tensor"
+            bl["gemm_frac_of_floor"] = t_floor[-1] * 1e6 / bl["gemm_us"]
+        hbm_dir = {
+            "store_gbs": st_r["gbs"], "load_gbs": ld_r["gbs"], "copy_gbs": hbm_peak,
+            "gemm_floor_us": sum(t_floor) * 1e6, "gemm_us": sum(gemm_ms) * 1e3,
+            "gemm_frac_of_floor": sum(t_floor) / (sum(gemm_ms) * 1e-3),
+            "what": "store-only and load-only rates of a grid-stride 16-byte kernel over 1 GiB (q8_measure_hbm_peak); per "
+                    "layer floor = max(2MNK / Int8 peak, 4MN / store-only rate)",
+        }
     emb_ms = t_emb / ksteps
     emb_bytes = 5.0 * M * H + 4.0 * M
     roofline = {
@@ -467,16 +561,18 @@ def run_ours(args):
         "frac_of_sustained_peak": achieved / int8_peak_sustained,
         "frac_of_nominal_4500": achieved / 4500.0,
         "int8_mma_issue_peak": mma_peak,
+        "hbm_one_directional": hbm_dir,
         "l2_sm_traffic": {
             "bytes_per_launch_mean": sum(fabric_bytes) / len(fabric_bytes),
             "achieved_tbs": sum(fabric_bytes) / (sum(gemm_ms) * 1e-3) / 1e12,
             "by_layer_tbs": {L["name"]: fb / (gm * 1e-3) / 1e12 for L, fb, gm in zip(layers, fabric_bytes, gemm_ms)},
-            "note": "operand re-loads of the 256 x 256 pair tiles plus the fp32 output, all through L2; the same kernel "
-                    "with its stores removed moves operands at about 10-11.7 TB/s, which is the limit it runs into",
+            "note": "operand re-loads of the 256 x 256 pair tiles plus the fp32 output, all through L2; with the epilogue "
+                    "left out the main loop alone moves operands at 12.6-12.9 TB/s (graph-replayed launches)",
         },
-        "note": "GEMM times: CUDA events around %d back-to-back launches of the layer (X_q just written by the quantise "
+        "note": "GEMM times: CUDA events around a graph replay of %d back-to-back launches of the layer (X_q just written by the quantise "
                 "pass, output streamed to HBM); quantise times: events around the back-to-back group of equal-sized layers "
-                "(a single launch for FFN2's input); embedding: events around its single launch (~4 us of overhead)" % GEMM_REPS,
+                "(a single launch for FFN2's input); embedding: events around %d launches that alternate between two output buffers; "
+                "all replayed from CUDA graphs unless --no-graph" % (GEMM_REPS, EMB_REPS),
         "by_layer": by_layer,
         "embedding": {"us": emb_ms * 1e3, "gbs": emb_bytes / (emb_ms * 1e-3) / 1e9,
                       "frac_hbm": emb_bytes / (emb_ms * 1e-3) / 1e9 / hbm_peak},
@@ -498,12 +594,13 @@ def run_ours(args):
             "sample": f"first {rows} of {M} token rows of each of the 4 FC layers, once ({dt:.1f} s)",
         }
 
+    graph_replayed = step_graph is not None
     # ---- whole encoder forwards (tokens/s): int8 embeddings, every FC quantised, attention / LayerNorm in fp32
     encoder = small = None
     if world == 1 and not args.no_encoder:
         for L in layers:
             L.clear()
-        del host_in, host_out, host_emb, emb_out
+        del host_in, host_out, host_emb, emb_out, emb_out2, gemm_graphs, quant_graphs, emb_graph, step_graph
         torch.cuda.empty_cache()
         encoder = measure_encoders(args, torch, q8)
         small = measure_small_cases(args, torch, q8)
@@ -518,6 +615,8 @@ def run_ours(args):
             "l2": "inputs larger than L2 (each step reads ~0.9 GB and writes ~1.0 GB; L2 is 126 MB)",
             "step": "q8_embedding + 4 x q8_linear (quantise, tcgen05 GEMM, fused epilogue), static scales",
             "streams": n_streams,
+            "launch": ("one CUDA graph replay per step" if graph_replayed else "eager launches"),
+            "eager_ms_per_step": eager_ms,
             "overlapped": (None if overlapped_ms is None else {
                 "streams": 5, "ms_per_step": overlapped_ms, "value": ops / (overlapped_ms * 1e-3) / 1e12, "unit": "TOPS",
                 "note": "same step, its five independent jobs on five streams (HBM-bound passes overlap the GEMMs)"}),
@@ -697,6 +796,7 @@ def main():
     ap.add_argument("--reference-rows", type=int, default=256, help="token rows per layer per step for --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-encoder", action="store_true", help="skip the whole-encoder tokens/s measurement")
+    ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of CUDA graph replays")
     ap.add_argument("--encoder-steps", type=int, default=5)
     ap.add_argument("--streams", type=int, default=1,
                     help="streams used inside a step for the independent layers of the FC set (1 = serial)")
