@@ -284,7 +284,7 @@ def run_ours(args):
     if not args.no_graph and not args.profile_mode and n_streams == 1:
         try:
             step_graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(step_graph):
+            with torch.cuda.graph(step_graph, capture_error_mode="thread_local"):
                 step()
             for _ in range(3):
                 step_graph.replay()
@@ -341,18 +341,18 @@ def run_ours(args):
             try:
                 for L in layers:
                     g = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(g):
+                    with torch.cuda.graph(g, capture_error_mode="thread_local"):
                         for _ in range(GEMM_REPS):
                             q8.q8_linear_q(L["Xq"], L["S_x"], L["Wq"], L["S_w"], L["bd"], L["act"], Y=L["Y"])
                     gemm_graphs.append(g)
                 for k, members in groups.items():
                     g = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(g):
+                    with torch.cuda.graph(g, capture_error_mode="thread_local"):
                         for i in members:
                             q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
                     quant_graphs[k] = g
                 emb_graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(emb_graph):
+                with torch.cuda.graph(emb_graph, capture_error_mode="thread_local"):
                     for r in range(EMB_REPS):
                         q8.q8_embedding(ids, Eq, S_e, out=emb_out if r % 2 == 0 else emb_out2)
                 torch.cuda.synchronize()
