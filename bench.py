@@ -594,7 +594,7 @@ def run_ours(args):
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
         from oracle import q8_oracle as o
-        rows = args.cpu_rows
+        rows = min(args.cpu_rows, M)
         t0 = time.perf_counter()
         for L in layers:
             Wq_h = L["Wq"].cpu().numpy()
@@ -804,7 +804,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=sorted(WORKLOADS), default="bert_large_fc")
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-rows", type=int, default=2048, help="token rows per layer for the cpu_baseline sample")
+    ap.add_argument("--cpu-rows", type=int, default=24576,
+                    help="token rows per layer for the cpu_baseline sample (default: the whole workload once, ~10 s)")
     ap.add_argument("--reference-rows", type=int, default=256, help="token rows per layer per step for --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-encoder", action="store_true", help="skip the whole-encoder tokens/s measurement")
