@@ -91,9 +91,16 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
     int8_t *Xq = static_cast<int8_t *>(workspace) + kWorkspaceHeaderBytes;
     Q8_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), s));
 
-    // Eq. 1, with the Sec. 4.1 dynamic scale when S_x is NULL (the header was just zeroed).
-    st = quantize_tensor(X, M * K, S_x, Xq, dbg_Xq, &hdr->S_x_dyn, true, &hdr->status, s);
-    if (st != Q8_OK) return st;
+    // Eq. 1, with the Sec. 4.1 dynamic scale when S_x is NULL (the header was just zeroed): the abs-max pass,
+    // then one kernel that turns the maximum into the scale and quantises with it.
+    if (S_x != nullptr) {
+        st = quantize_tensor(X, M * K, S_x, Xq, dbg_Xq, nullptr, true, &hdr->status, s);
+        if (st != Q8_OK) return st;
+    } else {
+        Q8_CUDA_TRY(launch_absmax(X, M * K, &hdr->absmax_bits, s));
+        Q8_CUDA_TRY(launch_quantize_dynamic(X, M * K, &hdr->absmax_bits, &hdr->S_x_dyn, &hdr->status, Xq, dbg_Xq, s));
+        last_launch_info().launches += 2;
+    }
 
     GemmArgs g;
     g.Xq = Xq;

@@ -97,12 +97,29 @@ __device__ __forceinline__ uint32_t quantize_pack4(float4 v, float S) { return q
 
 // VEC: a thread turns one 16-byte load (4 floats) into one 4-byte store, four of them in flight
 // per iteration; consecutive lanes touch consecutive addresses on both sides.
+// With absmax_bits (dynamic scale, Sec. 4.1) every thread derives S = 127 / max|x| from the finished abs-max word
+// itself (one correctly rounded division, the same value in every thread) and thread 0 of the grid publishes it
+// in *S_out for the GEMM that follows, so no separate scale kernel runs; otherwise S is read from S_ptr.
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restrict__ x, int64_t n,
                                                             const float *__restrict__ S_ptr,
-                                                            int8_t *__restrict__ xq, int8_t *__restrict__ xq_copy)
+                                                            int8_t *__restrict__ xq, int8_t *__restrict__ xq_copy,
+                                                            const uint32_t *__restrict__ absmax_bits = nullptr,
+                                                            float *__restrict__ S_out = nullptr,
+                                                            int32_t *__restrict__ status = nullptr)
 {
-    const float S = __ldg(S_ptr);
+    float S;
+    if (absmax_bits != nullptr) {
+        const float a = __uint_as_float(__ldg(absmax_bits));
+        const bool bad = !(a > 0.0f) || isinf(a);
+        S = bad ? 1.0f : __fdiv_rn(127.0f, a);
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            *S_out = S;
+            if (bad && status) atomicOr(status, 1 << Q8_ERR_SCALE);
+        }
+    } else {
+        S = __ldg(S_ptr);
+    }
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
     if (VEC) {
@@ -289,6 +306,20 @@ cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *x
         quantize_kernel<true><<<grid_for((n + 3) >> 2, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy);
     } else {
         quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *absmax_bits, float *S_out, int32_t *status,
+                                    int8_t *xq, int8_t *xq_copy, cudaStream_t s)
+{
+    if (n <= 0) return cudaSuccess;
+    if (aligned16(x) && aligned16(xq) && (xq_copy == nullptr || aligned16(xq_copy))) {
+        quantize_kernel<true><<<grid_for((n + 3) >> 2, kThreads * 4, 8), kThreads, 0, s>>>(x, n, nullptr, xq, xq_copy,
+                                                                                           absmax_bits, S_out, status);
+    } else {
+        quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, nullptr, xq, xq_copy, absmax_bits,
+                                                                                 S_out, status);
     }
     return cudaGetLastError();
 }

@@ -10,9 +10,10 @@ namespace q8 {
 
 // Layout of the head of a q8_linear workspace.
 struct WorkspaceHeader {
-    int32_t status;  // OR of (1 << q8_status) bits raised by kernels
-    float S_x_dyn;   // dynamic mode: first the float bits of max|X| (atomicMax scratch), then 127 / max|X|
-    int32_t pad[2];
+    int32_t status;        // OR of (1 << q8_status) bits raised by kernels
+    float S_x_dyn;         // dynamic mode: 127 / max|X|, written by the quantise kernel
+    uint32_t absmax_bits;  // dynamic mode: float bits of max|X| (atomicMax scratch, zero at the start of a call)
+    int32_t pad;
 };
 constexpr size_t kWorkspaceHeaderBytes = 256;
 
@@ -60,6 +61,10 @@ cudaError_t launch_absmax(const float *x, int64_t n, uint32_t *bits, cudaStream_
 cudaError_t launch_scale_from_absmax(const uint32_t *bits, float *S, int32_t *status, cudaStream_t s);
 cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy,
                             cudaStream_t s);
+// Eq. 1 with S = 127 / float(*absmax_bits) derived inside the kernel (dynamic scale); *S_out receives S and
+// *status the Q8_ERR_SCALE bit when the maximum is 0 or not finite (S = 1 then).  absmax_bits and S_out differ.
+cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *absmax_bits, float *S_out,
+                                    int32_t *status, int8_t *xq, int8_t *xq_copy, cudaStream_t s);
 cudaError_t launch_ema_update(CalibState *st, float decay, cudaStream_t s);
 cudaError_t launch_fake_quantize(const float *x, int64_t n, const float *S, float *xhat, cudaStream_t s);
 cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,

@@ -174,7 +174,7 @@ class Q8BertEncoder:
     def launches_per_forward(self, scales: str = "static", fused: bool = False) -> int:
         if fused:
             return 4 + self.L * 7
-        per_fc = 2 if scales == "static" else (4 if scales == "dynamic" else 6)
+        per_fc = 2 if scales == "static" else (3 if scales == "dynamic" else 5)
         return 4 + self.L * (4 * per_fc + 3)
 
     def poll(self):
