@@ -169,6 +169,30 @@ def test_int8_only_output_of_every_tile_shape(block_n, ctas, warps):
         q8.q8_tune_gemm_tile(0, 0)
 
 
+def test_int8_only_output_at_full_size():
+    """FFN1 of BERT-Large handing its GELU output to FFN2 as Int8 (M = 24576, automatic tile choice: CTA pairs,
+    staged TMA stores): equal to Eq. 1 applied to the fp32 output of the plain call, everywhere."""
+    K, N, act = 1024, 4096, 1
+    Xq = dev((synth.token_ids(M * K, 255, seed=1700) - 127).astype(np.int8).reshape(M, K))
+    Wq, S_w = q8.q8_quantize_weight(dev(synth.weight(N, K, seed=1701)))
+    bb = dev(synth.bias(N, seed=1702))
+    S_x = dev(np.array([4.25], np.float32))
+    S_y = dev(np.array([37.5], np.float32))
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Y = q8.q8_linear_q(Xq, S_x, Wq, S_w, bb, act, dev_status=st)
+    Yq = q8.q8_linear_q_requant(Xq, S_x, Wq, S_w, bb, act, S_y, dev_status=st)
+    info = q8.q8_last_launch_info()
+    assert q8.q8_poll_status(st) == (q8.Q8_OK, 0)
+    assert (info["gemm_kernel"], info["block_n"], info["ctas"]) == (1, 256, 2)
+    # row slabs through the oracle's Eq. 1 (first rows, rows across a tile boundary in the middle, last rows)
+    mid = (M // 2 // 256) * 256
+    for lo, hi in [(0, 64), (mid - 40, mid + 40), (M - 300, M)]:
+        assert np.array_equal(Yq[lo:hi].cpu().numpy(), o.quantize(Y[lo:hi].cpu().numpy(), 37.5))
+    # the whole tensor against Eq. 1 in plain torch ops on the device (secondary: one rounded fp32 multiply,
+    # nearest-even integer, symmetric clamp)
+    assert torch.equal(Yq, torch.clamp(torch.round(Y * 37.5), -127, 127).to(torch.int8))
+
+
 def test_hbm_peak_probe_runs_and_is_plausible():
     buf = torch.empty(1 << 29, dtype=torch.uint8, device="cuda")
     w = q8.q8_measure_hbm_peak(buf, store=True, repeats=5)
