@@ -193,6 +193,53 @@ def test_int8_only_output_at_full_size():
     assert torch.equal(Yq, torch.clamp(torch.round(Y * 37.5), -127, 127).to(torch.int8))
 
 
+def test_fused_qkv_with_per_layer_scales_at_full_size():
+    """BERT-Large Q, K and V as one [3072, 1024] matrix with one Eq. 3 scale per 1024-row layer, M = 24576, in the
+    benchmark's launch configuration (CTA pairs): row slabs equal three separate oracle layers."""
+    H = 1024
+    X = synth.activation(M, H, seed=1800)
+    Ws = [synth.normal((H, H), 0.02 * (1 + i), 1801 + i) for i in range(3)]
+    bs = [synth.bias(H, 1810 + i) for i in range(3)]
+    Wq, S_w = q8.q8_quantize_weight_segments(dev(np.concatenate(Ws)), H)
+    S_x = np.float32(4.5)
+    acc = torch.empty((M, 3 * H), dtype=torch.int32, device="cuda")
+    Y = q8.q8_linear_wseg(dev(X), Wq, S_w, H, dev(np.array([S_x], np.float32)), dev(np.concatenate(bs)), 0, dbg_acc=acc)
+    info = q8.q8_last_launch_info()
+    assert (info["gemm_kernel"], info["block_n"], info["ctas"]) == (1, 256, 2)
+    mid = (M // 2 // 256) * 256
+    for i in range(3):
+        Wq_ref, S_ref, _ = o.quantize_weight(Ws[i])
+        assert S_w[i].item() == S_ref and np.array_equal(Wq[i * H:(i + 1) * H].cpu().numpy(), Wq_ref)
+        for lo, hi in [(0, 40), (mid - 20, mid + 20), (M - 40, M)]:
+            ref = o.linear(X[lo:hi], Wq_ref, S_ref, S_x, bs[i], 0)
+            assert np.array_equal(acc[lo:hi, i * H:(i + 1) * H].cpu().numpy(), ref["acc"]), (i, lo)
+            err = np.abs(Y[lo:hi, i * H:(i + 1) * H].cpu().numpy().astype(np.float64) - ref["y"]).max()
+            assert err <= REL_TOL * np.abs(ref["y"]).max(), (i, lo, err)
+
+
+def test_every_tile_shape_gives_the_same_bits():
+    """The epilogue arithmetic of an output element does not depend on the tile it falls in: the fp32 output is
+    bit-identical across every instantiation of the tcgen05 kernel and the generic kernel's Int32 matrix."""
+    Mm, Nn, Kk = 1000, 520, 272
+    Xq = dev((synth.token_ids(Mm * Kk, 255, seed=1900) - 127).astype(np.int8).reshape(Mm, Kk))
+    Wq, S_w = q8.q8_quantize_weight(dev(synth.weight(Nn, Kk, seed=1901)))
+    bb = dev(synth.bias(Nn, seed=1902))
+    S_x = dev(np.array([5.5], np.float32))
+    outs = []
+    try:
+        for (bn, ctas, warps) in [(32, 1, 0), (64, 1, 0), (128, 1, 0), (256, 1, 0), (256, 2, 8), (256, 2, 16)]:
+            q8.q8_tune_gemm_tile(bn, ctas)
+            q8.q8_tune_gemm_epilogue_warps(warps)
+            for act in (0, 1):
+                acc = torch.empty((Mm, Nn), dtype=torch.int32, device="cuda")
+                outs.append((act, q8.q8_linear_q(Xq, S_x, Wq, S_w, bb, act, dbg_acc=acc), acc))
+    finally:
+        q8.q8_tune_gemm_epilogue_warps(0)
+        q8.q8_tune_gemm_tile(0, 0)
+    for act, Y, acc in outs[2:]:
+        assert torch.equal(Y, outs[act][1]) and torch.equal(acc, outs[act][2])
+
+
 def test_hbm_peak_probe_runs_and_is_plausible():
     buf = torch.empty(1 << 29, dtype=torch.uint8, device="cuda")
     w = q8.q8_measure_hbm_peak(buf, store=True, repeats=5)
