@@ -89,14 +89,14 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WorkspaceHeader *hdr = static_cast<WorkspaceHeader *>(workspace);
     int8_t *Xq = static_cast<int8_t *>(workspace) + kWorkspaceHeaderBytes;
-    Q8_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), s));
-
-    // Eq. 1, with the Sec. 4.1 dynamic scale when S_x is NULL (the header was just zeroed): the abs-max pass,
-    // then one kernel that turns the maximum into the scale and quantises with it.
+    // Eq. 1.  With a given scale the quantise kernel itself starts the call's status word at zero (no separate
+    // clearing operation in the stream); with the Sec. 4.1 dynamic scale (S_x NULL) the header is zeroed first, then
+    // come the abs-max pass and one kernel that turns the maximum into the scale and quantises with it.
     if (S_x != nullptr) {
-        st = quantize_tensor(X, M * K, S_x, Xq, dbg_Xq, nullptr, true, &hdr->status, s);
-        if (st != Q8_OK) return st;
+        Q8_CUDA_TRY(launch_quantize(X, M * K, S_x, Xq, dbg_Xq, s, &hdr->status));
+        last_launch_info().launches += 1;
     } else {
+        Q8_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), s));
         Q8_CUDA_TRY(launch_absmax(X, M * K, &hdr->absmax_bits, s));
         Q8_CUDA_TRY(launch_quantize_dynamic(X, M * K, &hdr->absmax_bits, &hdr->S_x_dyn, &hdr->status, Xq, dbg_Xq, s));
         last_launch_info().launches += 2;

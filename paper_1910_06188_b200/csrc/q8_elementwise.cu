@@ -106,8 +106,12 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                                                             int8_t *__restrict__ xq, int8_t *__restrict__ xq_copy,
                                                             const uint32_t *__restrict__ absmax_bits = nullptr,
                                                             float *__restrict__ S_out = nullptr,
-                                                            int32_t *__restrict__ status = nullptr)
+                                                            int32_t *__restrict__ status = nullptr,
+                                                            int32_t *__restrict__ clear_word = nullptr)
 {
+    grid_dependency_wait();
+    // first kernel of a static-scale q8_linear call: start the call's status word at zero
+    if (clear_word != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *clear_word = 0;
     float S;
     if (absmax_bits != nullptr) {
         const float a = __uint_as_float(__ldg(absmax_bits));
@@ -208,6 +212,7 @@ __global__ void __launch_bounds__(kThreads) embedding_kernel(const int32_t *__re
                                                              float *__restrict__ out, int8_t *__restrict__ rows_q,
                                                              int32_t *__restrict__ status)
 {
+    grid_dependency_wait();
     const float inv = __fdiv_rn(1.0f, __ldg(S_e));
     if (VEC) {
         const int per_row = (int)(H >> 2);
@@ -299,13 +304,16 @@ cudaError_t launch_scale_from_absmax(const uint32_t *bits, float *S, int32_t *st
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy, cudaStream_t s)
+cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy, cudaStream_t s,
+                            int32_t *clear_word)
 {
     if (n <= 0) return cudaSuccess;
     if (aligned16(x) && aligned16(xq) && (xq_copy == nullptr || aligned16(xq_copy))) {
-        quantize_kernel<true><<<grid_for((n + 3) >> 2, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy);
+        return launch_overlapping_tail(quantize_kernel<true>, dim3(grid_for((n + 3) >> 2, kThreads * 4, 8)), dim3(kThreads), 0, s,
+                                       x, n, S, xq, xq_copy, nullptr, nullptr, nullptr, clear_word);
     } else {
-        quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy);
+        quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy, nullptr, nullptr,
+                                                                                 nullptr, clear_word);
     }
     return cudaGetLastError();
 }
@@ -350,7 +358,8 @@ cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, co
         // one thread per 4-byte piece of a row, rounded up to whole warps; a CTA takes 4 rows per iteration
         int threads = (int)(((H >> 2) + 31) / 32 * 32);
         if (threads > kThreads) threads = kThreads;
-        embedding_kernel<true><<<grid_for((T + 3) / 4, 1, 16), threads, 0, s>>>(ids, T, Eq, S_e, V, H, out, rows_q, status);
+        return launch_overlapping_tail(embedding_kernel<true>, dim3(grid_for((T + 3) / 4, 1, 16)), dim3(threads), 0, s, ids, T,
+                                       Eq, S_e, V, H, out, rows_q, status);
     } else {
         embedding_kernel<false><<<grid_for(T * H, kThreads, 8), kThreads, 0, s>>>(ids, T, Eq, S_e, V, H, out,
                                                                                  rows_q, status);

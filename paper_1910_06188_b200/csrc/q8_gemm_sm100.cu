@@ -312,6 +312,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     if (CTAS == 2) cluster_sync_all();  // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only this CTA's own resources; the kernel before this one in the stream (which
+    // produced X_q) must be complete before anything below reads global memory
+    grid_dependency_wait();
 
     if (warp == 0) {
         // ---------------- TMA producer (each CTA loads its own rows) ----------------
@@ -665,13 +668,16 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = s;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = CTAS;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CTAS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    // set-up (barriers, TMEM) may overlap the tail of the preceding kernel; see grid_dependency_wait()
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     e = cudaLaunchKernelEx(&cfg, kernel, tx, tw, tw2, tw4, ty, tyq, a, tma_store, yq_tma, full_tiles, split);
     LaunchInfo &li = last_launch_info();
     li.gemm_kernel = 1;

@@ -59,8 +59,9 @@ LaunchInfo &last_launch_info();
 cudaError_t launch_absmax(const float *x, int64_t n, uint32_t *bits, cudaStream_t s);
 // *S = 127 / float(*bits) in place (bits and S may alias); flags Q8_ERR_SCALE on 0 / non-finite.
 cudaError_t launch_scale_from_absmax(const uint32_t *bits, float *S, int32_t *status, cudaStream_t s);
+// clear_word (may be NULL): a device word the kernel sets to zero before anything else (a call's status word).
 cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy,
-                            cudaStream_t s);
+                            cudaStream_t s, int32_t *clear_word = nullptr);
 // Eq. 1 with S = 127 / float(*absmax_bits) derived inside the kernel (dynamic scale); *S_out receives S and
 // *status the Q8_ERR_SCALE bit when the maximum is 0 or not finite (S = 1 then).  absmax_bits and S_out differ.
 cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *absmax_bits, float *S_out,
@@ -97,6 +98,30 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
                       float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
                       int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic, int8_t *Yq = nullptr,
                       const float *S_y = nullptr, int64_t w_seg = 0);
+
+// ---- programmatic dependent launch
+// A kernel launched with launch_overlapping_tail() may be scheduled while the kernel before it in the stream is
+// still draining (its last CTAs finishing), so that its own start-up overlaps that tail.  Such a kernel must call
+// grid_dependency_wait() before its first global-memory access: the call returns once the preceding kernel has
+// completed and its writes are visible (and at once when the kernel was launched the ordinary way).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapping_tail(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // Eq. 1 on one value: one rounded fp32 multiply, nearest-even integer (NaN -> 0, saturating), symmetric clamp.
 __device__ __forceinline__ int32_t quantize_value(float x, float S)

@@ -48,7 +48,7 @@ extern "C" q8_status q8_linear_noalloc(const float *X, const int8_t *Wq, const f
     q8_status st = static_scratch(&scratch);
     if (st != Q8_OK) return st;
     if (status_word) *status_word = scratch;  // the status word sits at offset 0 of the scratch
-    // linear_impl clears the header (status word, dynamic-scale word) at the start of every call and
+    // linear_impl starts the status word (and, with a dynamic scale, the scale words) at zero in every call and
     // overwrites the quantised activation, so nothing of the previous call's contents is read.
     return q8::linear_impl(X, Wq, S_w, S_x, bias, act, Y, M, N, K, scratch, kStaticScratchBytes, dbg_Xq, dbg_acc,
                            stream, false);
