@@ -126,6 +126,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     const uint32_t tmem_o = tmem_base + (uint32_t)s_pad;  // O_main: 64 columns behind the scores; O_corr: the next 64
+    grid_dependency_wait();  // the set-up above may overlap the tail of the kernel that produced qkv
 
     if (warp == kWorkers / 32) {
         // ================= MMA warp: one lane issues, chunk after chunk, as the workers report operands ready
@@ -404,9 +405,8 @@ cudaError_t launch_attention_tc(const float *qkv, int64_t B, int64_t S, int64_t 
     while (cols < (uint32_t)(s_pad + 2 * kHeadDim)) cols <<= 1;  // scores, O_main, O_corr
     dim3 grid((unsigned)((S + kQTile - 1) / kQTile), (unsigned)heads, (unsigned)B);
     const float scale = 1.4426950408889634f / 8.0f;  // log2(e) / sqrt(64): the softmax then uses 2^x
-    attention_tc_kernel<<<grid, kThreads, kAttnTcSmemBytes, s>>>(qkv, (int)S, heads * kHeadDim, scale, ctx, S_q, ctx_q, cols,
-                                                                 attention_status_word());
-    return cudaGetLastError();
+    return launch_overlapping_tail(attention_tc_kernel, grid, dim3(kThreads), kAttnTcSmemBytes, s, qkv, (int)S,
+                                   heads * kHeadDim, scale, ctx, S_q, ctx_q, cols, attention_status_word());
 }
 
 }  // namespace q8

@@ -134,6 +134,7 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_warp_kernel(const fl
                                                                         const float *__restrict__ S_q,
                                                                         int8_t *__restrict__ out_q)
 {
+    grid_dependency_wait();  // launched so that its start may overlap the tail of the kernel before it
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (kLnThreads / 32) + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -350,7 +351,8 @@ cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r
                      al16(beta) && al16(out) && (reinterpret_cast<uintptr_t>(out_q) & 3u) == 0;
     if (vec && H <= 1024) {
         const unsigned blocks = (unsigned)((rows + kLnThreads / 32 - 1) / (kLnThreads / 32));
-        add_layernorm_warp_kernel<<<blocks, kLnThreads, 0, s>>>(x, r1, r2, gamma, beta, eps, rows, H, out, S_q, out_q);
+        return launch_overlapping_tail(add_layernorm_warp_kernel, dim3(blocks), dim3(kLnThreads), 0, s, x, r1, r2, gamma, beta,
+                                       eps, rows, H, out, S_q, out_q);
     } else if (vec) {
         add_layernorm_vec_kernel<<<(unsigned)rows, kLnThreads, 0, s>>>(x, r1, r2, gamma, beta, eps, H, out, S_q, out_q);
     } else {
