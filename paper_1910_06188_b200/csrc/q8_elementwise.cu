@@ -323,8 +323,8 @@ cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *a
 {
     if (n <= 0) return cudaSuccess;
     if (aligned16(x) && aligned16(xq) && (xq_copy == nullptr || aligned16(xq_copy))) {
-        quantize_kernel<true><<<grid_for((n + 3) >> 2, kThreads * 4, 8), kThreads, 0, s>>>(x, n, nullptr, xq, xq_copy,
-                                                                                           absmax_bits, S_out, status);
+        return launch_overlapping_tail(quantize_kernel<true>, dim3(grid_for((n + 3) >> 2, kThreads * 4, 8)), dim3(kThreads), 0, s,
+                                       x, n, nullptr, xq, xq_copy, absmax_bits, S_out, status, nullptr);
     } else {
         quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, nullptr, xq, xq_copy, absmax_bits,
                                                                                  S_out, status);
