@@ -530,20 +530,59 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
+// A tensor map depends only on the base address, the extents and the box, and a serving loop calls with the same
+// few buffers over and over, so the encoded maps are kept in a small per-thread table (direct-mapped on a hash of
+// those fields): a hit saves the driver call, which matters for launch-bound small problems.
+struct TmapKey {
+    const void *base;
+    int64_t d0, d1;
+    int32_t box0, box1, kind;
+    bool operator==(const TmapKey &o) const
+    {
+        return base == o.base && d0 == o.d0 && d1 == o.d1 && box0 == o.box0 && box1 == o.box1 && kind == o.kind;
+    }
+};
+struct TmapSlot {
+    TmapKey key;
+    CUtensorMap map;
+    bool valid = false;
+};
+constexpr int kTmapSlots = 64;
+
+template <typename Encode>
+bool cached_tmap(CUtensorMap *out, const TmapKey &key, Encode encode)
+{
+    static thread_local TmapSlot table[kTmapSlots];
+    uint64_t h = reinterpret_cast<uintptr_t>(key.base) * 0x9E3779B97F4A7C15ull;
+    h ^= (uint64_t)key.d0 * 0xC2B2AE3D27D4EB4Full + (uint64_t)key.d1 * 0x165667B19E3779F9ull +
+         (uint64_t)(key.box1 * 131 + key.box0 * 7 + key.kind);
+    TmapSlot &slot = table[(h >> 40) % kTmapSlots];
+    if (slot.valid && slot.key == key) {
+        *out = slot.map;
+        return true;
+    }
+    if (!encode(out)) return false;
+    slot.key = key;
+    slot.map = *out;
+    slot.valid = true;
+    return true;
+}
+
 // Row-major int8 matrix [rows, K] as a 2-D tensor map with (128 x box_rows) boxes, 128-byte swizzle.
 // Elements outside the matrix read as zero, which is what ragged M, N and K tails need.
 bool make_tmap(CUtensorMap *map, const int8_t *base, int64_t rows, int64_t K, int box_rows)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)K};
-    cuuint32_t box[2] = {(cuuint32_t)BLOCK_K, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return cached_tmap(map, TmapKey{base, K, rows, BLOCK_K, box_rows, 0}, [&](CUtensorMap *m) {
+        cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+        cuuint64_t strides[1] = {(cuuint64_t)K};
+        cuuint32_t box[2] = {(cuuint32_t)BLOCK_K, (cuuint32_t)box_rows};
+        cuuint32_t estr[2] = {1, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 // Row-major fp32 output [M, N] as a tensor map of 32 x 32 boxes (128 bytes wide), 128-byte swizzle.
@@ -552,14 +591,15 @@ bool make_tmap_out(CUtensorMap *map, float *base, int64_t M, int64_t N)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-    cuuint64_t strides[1] = {(cuuint64_t)N * 4};
-    cuuint32_t box[2] = {32, 32};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return cached_tmap(map, TmapKey{base, N, M, 32, 32, 1}, [&](CUtensorMap *m) {
+        cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+        cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+        cuuint32_t box[2] = {32, 32};
+        cuuint32_t estr[2] = {1, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 // Row-major Int8 output [M, N] as a tensor map of (box_cols x 32) boxes: 64-byte rows with the 64-byte swizzle
@@ -568,14 +608,15 @@ bool make_tmap_out_q(CUtensorMap *map, int8_t *base, int64_t M, int64_t N, int b
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-    cuuint64_t strides[1] = {(cuuint64_t)N};
-    cuuint32_t box[2] = {(cuuint32_t)box_cols, 32};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    box_cols == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    return cached_tmap(map, TmapKey{base, N, M, box_cols, 32, 2}, [&](CUtensorMap *m) {
+        cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+        cuuint64_t strides[1] = {(cuuint64_t)N};
+        cuuint32_t box[2] = {(cuuint32_t)box_cols, 32};
+        cuuint32_t estr[2] = {1, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  box_cols == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 int sm_count()
