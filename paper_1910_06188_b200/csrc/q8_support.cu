@@ -15,6 +15,7 @@ namespace {
 // One CTA per row.  The summed row is kept in shared memory, so the inputs are read once; mean and
 // variance are the two-pass forms (sum, then sum of squared deviations), reduced through warp shuffles.
 constexpr int kLnThreads = 256;
+constexpr int kLnCtasPerSm = 4;  // CTAs per SM of the warp-per-row kernel (64 registers x 256 threads each)
 
 __device__ __forceinline__ float block_sum(float v, float *scratch)
 {
@@ -136,9 +137,11 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_warp_kernel(const fl
 {
     grid_dependency_wait();  // launched so that its start may overlap the tail of the kernel before it
     const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * (kLnThreads / 32) + (threadIdx.x >> 5);
-    if (row >= rows) return;
     const int n4 = (int)(H >> 2);
+    const float Sq = out_q ? __ldg(S_q) : 1.0f;
+    // the grid is sized to the device and every warp walks rows with a grid stride (no partial last wave)
+    for (int64_t row = (int64_t)blockIdx.x * (kLnThreads / 32) + (threadIdx.x >> 5); row < rows;
+         row += (int64_t)gridDim.x * (kLnThreads / 32)) {
     const int64_t base4 = row * n4;
     const float4 *x4 = reinterpret_cast<const float4 *>(x) + base4;
     const float4 *a4 = r1 ? reinterpret_cast<const float4 *>(r1) + base4 : nullptr;
@@ -169,7 +172,6 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_warp_kernel(const fl
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
     const float rstd = 1.0f / sqrtf(q / (float)H + eps);
-    const float Sq = out_q ? __ldg(S_q) : 1.0f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int c = lane + 32 * i;
@@ -183,6 +185,7 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_warp_kernel(const fl
         y.w = (v[i].w - mean) * rstd * g.w + b.w;
         if (out) reinterpret_cast<float4 *>(out)[base4 + c] = y;
         if (out_q) reinterpret_cast<uint32_t *>(out_q)[base4 + c] = quantize_pack4(y.x, y.y, y.z, y.w, Sq);
+    }
     }
 }
 
@@ -350,7 +353,11 @@ cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r
     const bool vec = (H % 4 == 0) && H <= 4 * 4 * kLnThreads && al16(x) && al16(r1) && al16(r2) && al16(gamma) &&
                      al16(beta) && al16(out) && (reinterpret_cast<uintptr_t>(out_q) & 3u) == 0;
     if (vec && H <= 1024) {
-        const unsigned blocks = (unsigned)((rows + kLnThreads / 32 - 1) / (kLnThreads / 32));
+        const int64_t want = (rows + kLnThreads / 32 - 1) / (kLnThreads / 32);
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int64_t cap = (int64_t)(sms > 0 ? sms : 148) * kLnCtasPerSm;
+        const unsigned blocks = (unsigned)(want < cap ? want : cap);
         return launch_overlapping_tail(add_layernorm_warp_kernel, dim3(blocks), dim3(kLnThreads), 0, s, x, r1, r2, gamma, beta,
                                        eps, rows, H, out, S_q, out_q);
     } else if (vec) {
