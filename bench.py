@@ -781,6 +781,27 @@ def measure_encoders(args, torch, q8):
         for key, a0, a1 in evs:
             shares[key] += a0.elapsed_time(a1)
         fc_ops = enc.L * sum(2.0 * T * N * K for _, K, N, _ in synth.fc_set(enc.H, enc.F))
+        # CPU oracle beside it (part of the cpu_baseline leg): one encoder layer of this model on one sequence
+        # (batch 1), timed on the host cores and extrapolated linearly to the whole model.
+        cpu_oracle = None
+        if not args.no_cpu_baseline:
+            from oracle import q8_oracle as o
+            f32 = lambda a: np.asarray(a, dtype=np.float32)
+            lw = {n: (enc.layers[0][n]["Wq"].cpu().numpy(), float(enc.layers[0][n]["S_w"].item()),
+                      float(q8.calibrate_S_x(enc.layers[0][n]["state"]).item()), enc.layers[0][n]["b"].cpu().numpy())
+                  for n in ("qkv", "attn_out", "ffn1", "ffn2")}
+            h = synth.activation(S, enc.H, synth.seed_for(cfg, 95))
+            lin = lambda n, X, act: f32(o.linear(X, lw[n][0], lw[n][1], lw[n][2], lw[n][3], act)["y"])
+            t0 = time.perf_counter()
+            qkv = lin("qkv", h, 0)
+            ctx = f32(o.attention(qkv, 1, S, enc.heads))
+            h1 = f32(o.add_layernorm(lin("attn_out", ctx, 0), h, eps=enc_mod.LN_EPS))
+            f2 = lin("ffn2", lin("ffn1", h1, 1), 0)
+            o.add_layernorm(f2, h1, eps=enc_mod.LN_EPS)
+            dt = time.perf_counter() - t0
+            cpu_oracle = {"one_layer_one_sequence_s": dt, "tokens_per_s_extrapolated": S / (dt * enc.L),
+                          "cores": os.cpu_count(), "kind": "oracle",
+                          "sample": f"layer 0 on one sequence of {S} tokens; extrapolated linearly to {enc.L} layers"}
         out[name] = {
             "tokens_per_s": T / (ms * 1e-3), "ms_per_forward": ms, "layers": enc.L, "tokens": T,
             "tokens_per_s_fused_requant": T / (ms_fused * 1e-3), "ms_per_forward_fused_requant": ms_fused,
@@ -790,6 +811,7 @@ def measure_encoders(args, torch, q8):
             "status": [list(c) for c in codes],
             "ms_by_kind": shares, "q8_linear_tops_inside_forward": fc_ops / (shares["q8_linear"] * 1e-3) / 1e12,
             "int8_parameter_bytes": enc.memory_bytes_int8(),
+            "cpu_oracle": cpu_oracle,
         }
         del enc
         torch.cuda.empty_cache()
