@@ -130,10 +130,17 @@ __device__ __forceinline__ int32_t quantize_value(float x, float S)
     return max(-127, min(127, q));
 }
 
+// Four values of Eq. 1 packed little-endian (a in the lowest byte).  The lower clamp is an integer max; the upper
+// clamp and the packing are done by cvt.pack.sat.s8.s32, which saturates each Int32 to [-128, 127] while it packs
+// two of them into the low half of the result and moves the low half of its third operand into the high half.
 __device__ __forceinline__ uint32_t quantize_pack4(float a, float b, float c, float d, float S)
 {
-    return ((uint32_t)quantize_value(a, S) & 0xffu) | (((uint32_t)quantize_value(b, S) & 0xffu) << 8) |
-           (((uint32_t)quantize_value(c, S) & 0xffu) << 16) | (((uint32_t)quantize_value(d, S) & 0xffu) << 24);
+    const int32_t qa = max(__float2int_rn(__fmul_rn(a, S)), -127), qb = max(__float2int_rn(__fmul_rn(b, S)), -127);
+    const int32_t qc = max(__float2int_rn(__fmul_rn(c, S)), -127), qd = max(__float2int_rn(__fmul_rn(d, S)), -127);
+    uint32_t hi, r;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(qd), "r"(qc), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(qb), "r"(qa), "r"(hi));
+    return r;
 }
 
 // ---- epilogue arithmetic shared by both GEMM kernels ----
