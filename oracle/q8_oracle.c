@@ -59,10 +59,12 @@ float q8o_scale_from_absmax(float absmax, int *flag)
 }
 
 /* Eq. 4: running EMA of max|x| over calibration batches.
- * state: ema[0] (fp32), n[0] (batches seen).  Returns S_x = M / ema. */
+ * state: ema[0] (fp32), n[0] (batches seen).  Returns S_x = M / ema.
+ * decay == 0 keeps no history: the EMA is the maximum of this batch itself, i.e. the scale is exactly
+ * the dynamic scale of Sec. 4.1 (no rounding from the update formula). */
 float q8o_ema_update(float *ema, int32_t *n, float batch_absmax, float decay, int *flag)
 {
-    if (*n == 0) {
+    if (*n == 0 || decay == 0.0f) {
         *ema = batch_absmax;
     } else {
         float one_minus_d = 1.0f - decay;
@@ -72,6 +74,14 @@ float q8o_ema_update(float *ema, int32_t *n, float batch_absmax, float decay, in
     }
     *n += 1;
     return q8o_scale_from_absmax(*ema, flag);
+}
+
+/* Eq. 4 on one calibration batch x of `numel` values.  An empty batch carries no observation of max|x|:
+ * the state is left as it is and the current scale is returned (1 before any batch has been seen). */
+float q8o_calibrate_batch(float *ema, int32_t *n, const float *x, int64_t numel, float decay, int *flag)
+{
+    if (numel <= 0) return *n == 0 ? 1.0f : q8o_scale_from_absmax(*ema, flag);
+    return q8o_ema_update(ema, n, q8o_absmax(x, numel), decay, flag);
 }
 
 /* Eq. 1 with Eq. 2 at b = 8: Quantize(x | S, M) = Clamp(nint(x*S), -M, M). */
@@ -134,7 +144,7 @@ void q8o_quantize_bias(const float *b, int64_t N, float S_x, float S_w, int32_t 
     }
 }
 
-/* "accumulated to the Int32 bias": acc[m][n] += b_q[n] in Int32.  Returns how many sums left
+/* Sec. 3, inference mode, the Int32 bias add: acc[m][n] += b_q[n] in Int32.  Returns how many sums left
  * the int32 range (they are wrapped to two's complement, as 32-bit hardware would). */
 int64_t q8o_add_bias(int32_t *acc, const int32_t *bq, int64_t M, int64_t N)
 {

@@ -43,6 +43,8 @@ def lib() -> C.CDLL:
         L.q8o_scale_from_absmax.argtypes = [C.c_float, ip]
         L.q8o_ema_update.restype = C.c_float
         L.q8o_ema_update.argtypes = [fp, i32p, C.c_float, C.c_float, ip]
+        L.q8o_calibrate_batch.restype = C.c_float
+        L.q8o_calibrate_batch.argtypes = [fp, i32p, fp, C.c_int64, C.c_float, ip]
         L.q8o_quantize.restype = None
         L.q8o_quantize.argtypes = [fp, C.c_int64, C.c_float, i8p]
         L.q8o_quantize_weight.restype = C.c_float
@@ -118,6 +120,16 @@ class EmaState:
         s = lib().q8o_ema_update(_p(self.ema, C.c_float), _p(self.n, C.c_int32),
                                  C.c_float(float(np.float32(batch_absmax))),
                                  C.c_float(float(np.float32(decay))), C.byref(flag))
+        self.S_x = np.float32(s)
+        self.flag |= int(flag.value)
+        return self.S_x
+
+    def update_batch(self, x, decay) -> np.float32:
+        """Eq. 4 on one calibration batch given as a tensor (an empty batch changes nothing)."""
+        x = _f32(x).ravel()
+        flag = C.c_int(0)
+        s = lib().q8o_calibrate_batch(_p(self.ema, C.c_float), _p(self.n, C.c_int32), _p(x, C.c_float), x.size,
+                                      C.c_float(float(np.float32(decay))), C.byref(flag))
         self.S_x = np.float32(s)
         self.flag |= int(flag.value)
         return self.S_x

@@ -17,7 +17,15 @@ MUTANTS = {
     "clamp_at_128": ("return ((int64_t)1 << (b - 1)) - 1;", "return ((int64_t)1 << (b - 1));"),
     "weight_transposed": ("s += (int64_t)xq[m * K + k] * (int64_t)wq[n * K + k];", "s += (int64_t)xq[m * K + k] * (int64_t)wq[k * N + n];"),
     "ema_wrong_sign": ("*ema = *ema + step;", "*ema = *ema - step;"),
-    "ema_zero_init": ("    if (*n == 0) {\n        *ema = batch_absmax;\n    } else {", "    if (0) {\n        *ema = batch_absmax;\n    } else {"),
+    "ema_zero_init": ("    if (*n == 0 || decay == 0.0f) {\n        *ema = batch_absmax;\n    } else {", "    if (0) {\n        *ema = batch_absmax;\n    } else {"),
+    "bias_ties_away": ("double r = (double)rintf(p);", "double r = (double)roundf(p);"),
+    "bias_product_in_double": ("float S_out = S_x * S_w;\n    double M32", "double S_out = (double)S_x * (double)S_w;\n    double M32"),
+    "bias_add_drops_overflow_count": ("            if (s > INT32_MAX || s < INT32_MIN) bad += 1;\n            acc[m * N + n] = (int32_t)(uint32_t)(uint64_t)s;",
+                                      "            acc[m * N + n] = (int32_t)(uint32_t)(uint64_t)s;"),
+    "bias_add_saturates": ("            acc[m * N + n] = (int32_t)(uint32_t)(uint64_t)s;",
+                           "            acc[m * N + n] = s > INT32_MAX ? INT32_MAX : (s < INT32_MIN ? INT32_MIN : (int32_t)s);"),
+    "ema_decay_zero_uses_update_formula": ("if (*n == 0 || decay == 0.0f) {", "if (*n == 0) {"),
+    "empty_batch_counts_as_zero_maximum": ("if (numel <= 0) return *n == 0 ? 1.0f : q8o_scale_from_absmax(*ema, flag);", ""),
     "bias_without_weight_scale": ("float S_out = S_x * S_w;\n    double M32", "float S_out = S_x;\n    double M32"),
     "dequant_by_sum_of_scales": ("double denom = (double)S_x * (double)S_w;", "double denom = (double)S_x + (double)S_w;"),
     "gelu_without_half": ("y[i] = 0.5 * y[i] * (1.0 + erf(y[i] * inv_sqrt2));", "y[i] = y[i] * (1.0 + erf(y[i] * inv_sqrt2));"),

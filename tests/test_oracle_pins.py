@@ -165,10 +165,26 @@ def test_ema_fixed_point_and_dynamic_limit():
     for m in (5.0, 0.25, 9.0):
         st.update(m, 0.0)                                     # decay 0: the EMA is the last maximum
     assert st.ema[0] == np.float32(9.0)
+    # ... exactly, also where ema + 1*(m - ema) would not give m back in fp32 (Sec. 4.1: the dynamic scale)
+    st = o.EmaState()
+    for m in (np.float32(1e8), np.float32(0.3), np.float32(3.0000002), np.float32(1.1)):
+        S = st.update(m, 0.0)
+        assert st.ema[0] == m and S == np.float32(127.0) / m
+    assert np.float32(1e8) + (np.float32(0.3) - np.float32(1e8)) != np.float32(0.3)   # the update formula would give 0
     st = o.EmaState()
     st.update(4.0, 0.9999)
     st.update(8.0, 0.9999)
     assert 4.0 < st.ema[0] < 4.001                            # moves towards the new maximum, slowly
+
+
+def test_empty_calibration_batch_changes_nothing():
+    st = o.EmaState()
+    assert st.update_batch(np.zeros(0, np.float32), 0.9) == np.float32(1.0) and int(st.n[0]) == 0 and st.flag == 0
+    x = np.array([0.5, -4.0, 1.0], np.float32)
+    S = st.update_batch(x, 0.9)
+    assert S == np.float32(127.0) / np.float32(4.0) and int(st.n[0]) == 1
+    assert st.update_batch(np.zeros(0, np.float32), 0.9) == S and int(st.n[0]) == 1 and st.ema[0] == np.float32(4.0)
+    assert st.update_batch(np.array([2.0], np.float32), 0.5) == np.float32(127.0) / np.float32(3.0)
 
 
 # ---------------------------------------------------------------- bias, dequantise, GELU
@@ -185,6 +201,34 @@ def test_bias_hand_example(pins):
 def test_bias_clamps_at_int32_M():
     bq = o.quantize_bias(np.array([1e30, -1e30, 0.0], np.float32), 4.0, 1000.0)
     assert bq.tolist() == [2 ** 31 - 1, -(2 ** 31 - 1), 0]
+
+
+def test_bias_ties_round_half_to_even(pins):
+    g = pins["bias_ties"]
+    bq = o.quantize_bias(np.array(g["b"], np.float32), g["S_x"], g["S_w"])
+    assert bq.tolist() == g["bq"]
+    assert bq.tolist() != g["bq_if_half_away"]
+
+
+def test_bias_scale_product_is_rounded_to_fp32_first(pins):
+    g = pins["bias_product_fp32"]
+    bq = o.quantize_bias(np.array([g["b"], -g["b"]], np.float32), g["S_x"], g["S_w"])
+    assert bq.tolist() == [g["bq"], -g["bq"]]
+    assert g["bq"] != g["bq_if_product_unrounded"]
+
+
+def test_bias_add_wraps_and_counts(pins):
+    g = pins["bias_add_wraps"]
+    acc, bad = o.add_bias(np.array(g["acc"], np.int32), np.array(g["bq"], np.int32))
+    assert acc.tolist() == g["sum"] and bad == g["overflows"]
+    # the whole layer reports the same condition: a saturated K = 133144 row plus a bias that tips it over
+    K = 133144
+    X = np.full((1, K), 127.0, np.float32)
+    Wq = np.full((1, K), 127, np.int8)
+    r = o.linear(X, Wq, 1.0, 1.0, np.array([5000.0], np.float32), 0)
+    assert r["flags"] & 2 and r["acc"][0, 0] == 16129 * K + 5000 - 2 ** 32
+    r = o.linear(X, Wq, 1.0, 1.0, np.array([4000.0], np.float32), 0)
+    assert r["flags"] == 0 and r["acc"][0, 0] == 16129 * K + 4000
 
 
 def test_gelu_textbook_values(pins):
