@@ -65,6 +65,7 @@ q8_status q8_quantize_weight(const float *W, int64_t N, int64_t K, int8_t *Wq, f
 
 /* Eq. 1 on an activation tensor (flat, `numel` elements).
  *   S_x != NULL: static scale (an Eq. 4 result), read.           S_x_used may be NULL.
+ *                A value that is not a positive finite number flags Q8_ERR_SCALE in dev_status.
  *   S_x == NULL: dynamic scale of Sec. 4.1, S = 127 / max|X| over this tensor, written to
  *                S_x_used (required; it also serves as the reduction scratch word).
  *   Xq     int8 [numel], written. */
@@ -75,8 +76,9 @@ q8_status q8_quantize_activation(const float *X, int64_t numel, const float *S_x
  * zero-initialised device block laid out as
  *   { float ema; float S_x; int32 n_batches; uint32 scratch; int32 status; int32 pad[3]; }
  * The first batch sets ema = max|X|; later ones do ema += (1 - decay) * (max|X| - ema) in fp32;
- * then S_x = 127 / ema.  decay must lie in [0, 1); decay 0 tracks the last batch (the dynamic scale, up to one fp32 rounding).
- * &state->S_x can be passed as S_x to q8_linear. */
+ * then S_x = 127 / ema.  decay must lie in [0, 1); decay 0 keeps no history: ema is exactly this batch's
+ * max|X| and S_x exactly the dynamic scale of Sec. 4.1.  A batch with numel == 0 carries no observation and
+ * leaves the state untouched (nothing is launched).  &state->S_x can be passed as S_x to q8_linear. */
 q8_status q8_calibrate(const float *X, int64_t numel, float decay, void *state, void *stream);
 size_t q8_calibrate_state_bytes(void);
 
@@ -94,7 +96,8 @@ q8_status q8_ste_backward(const float *grad_out, int64_t numel, float *grad_in, 
  *   b_q = Clamp(nint(b * fl32(S_x * S_w)), -(2^31-1), 2^31-1);  Y = (acc + b_q) / (S_x * S_w);
  *   optional GELU.
  *   X [M,K] fp32; Wq [N,K] int8 with its scale S_w (from q8_quantize_weight); bias [N] fp32 or NULL.
- *   S_x: static activation scale, or NULL for the dynamic scale 127 / max|X| of Sec. 4.1.
+ *   S_x: static activation scale, or NULL for the dynamic scale 127 / max|X| of Sec. 4.1.  A static scale
+ *     that is not a positive finite number flags Q8_ERR_SCALE in the status word (the output is then meaningless).
  *   act: Q8_ACT_NONE or Q8_ACT_GELU.      Y [M,N] fp32, written.
  *   workspace: >= q8_linear_workspace_bytes(M,N,K) bytes, 256-byte aligned, caller-owned scratch
  *     (status word at offset 0, then the quantised activation).  Its contents need not be
@@ -131,7 +134,10 @@ q8_status q8_linear_generic(const float *X, const int8_t *Wq, const float *S_w, 
  * whose allocator is frozen after initialisation.  It computes exactly what q8_linear computes, with
  * the same arguments minus the workspace: the scratch (status word + Int8 activation) is a fixed
  * array inside the library image, present on every GPU that loads the library until the process
- * exits.  The call itself performs no allocation of any kind.
+ * exits.  Once the library is warm on a device the call performs no allocation of any kind; the very
+ * first call on a device (and the first use of each GEMM tile configuration) makes the CUDA runtime load
+ * the kernels and the array there, so issue one warm-up call per device and shape class at start-up.
+ * The looked-up addresses are cached per device and do not survive cudaDeviceReset.
  *   Limit: M * K <= Q8_NOALLOC_MAX_MK (16 Mi elements, i.e. 16 MiB of scratch + a 256-byte header);
  *     larger activations are refused with Q8_ERR_WORKSPACE before anything is launched.
  *   status_word (host pointer, may be NULL) receives the device address of the status word, which
@@ -217,60 +223,14 @@ const char *q8_status_string(q8_status s);
  * any pointer may be NULL. */
 void q8_last_launch_info(int *gemm_kernel, int *launches, int *block_n, int *grid, int *ctas);
 
-/* Tuning / test hook: force the tile shape of the tcgen05 GEMM for later calls in this process.
- * (block_n, ctas) = (0, 0) restores the automatic choice; otherwise ctas = 1 with block_n in
- * {32, 64, 128, 256} (one SM per 128 x block_n tile) or ctas = 2 with block_n = 256 (a pair of
- * SMs per 256 x 256 tile).  Results do not depend on the choice.  Not thread-safe. */
-q8_status q8_tune_gemm_tile(int block_n, int ctas);
-
-/* Tuning / test hook: epilogue warps per CTA of the cta_group::2 kernel for later calls in this process:
- * 8 (each warp pipelines four 32-column blocks per tile through two staging buffers), 16 (two blocks per
- * warp, one staging buffer) or 0 = automatic.  Other values are Q8_ERR_ARG.  Results do not depend on it. */
-q8_status q8_tune_gemm_epilogue_warps(int warps);
-
-/* Tuning / test hook for the schedule of the cta_group::2 kernel.  When the number of 256 x 256 tiles
- * is not a multiple of the number of SM pairs, the tiles of the last, partial round are cut into 2 or 4
- * narrower tiles (256 x 128 or 256 x 64) if these still fit in one round, which shortens that round.
- * enable = 0 switches this off for later calls in this process, non-zero (the default) on.  Results do
- * not depend on it.  Not thread-safe.  (An implementation detail with no counterpart in the paper.) */
-void q8_tune_gemm_tail_split(int enable);
-
-/* Into how many narrower tiles each tile of the last round was cut by the most recent tcgen05 GEMM launch
- * of this host thread: 1 (not cut), 2 or 4. */
-int q8_last_launch_tail_split(void);
-
 /* q8_attention / q8_attention_quant run on the tensor cores when the padded sequence fits the accumulator
  * memory (S rounded up to a multiple of 64, plus 64, at most 512 columns: S <= 448) and the pointers are
  * 16-byte aligned: both products as tcgen05.mma kind::tf32 on operands split into a TF32-exact high part and a
- * low remainder, three partial products accumulated in fp32, which keeps fp32-grade accuracy.  Otherwise, or
- * after q8_tune_attention(0), a CUDA-core fp32 kernel computes the same thing.  The tensor-core kernel bounds
+ * low remainder, three partial products accumulated in fp32, which keeps fp32-grade accuracy.  Otherwise a
+ * CUDA-core fp32 kernel computes the same thing.  The tensor-core kernel bounds
  * its waits; a time-out sets the Q8_ERR_TIMEOUT bit in a per-device status word whose device address
- * q8_attention_status_word returns (poll it with q8_poll_status).  Not thread-safe. */
-void q8_tune_attention(int use_tensor_cores);
+ * q8_attention_status_word returns (poll it with q8_poll_status). */
 q8_status q8_attention_status_word(void **dev_status);
-
-/* Measurement aid, no counterpart in the paper: the issue-bound Int8 rate of the tensor cores of the current
- * device, i.e. the ceiling of the GEMM's tensor pipe when operands cost nothing.  Every SM (ctas = 1) or SM
- * pair (ctas = 2, cta_group::2) issues the GEMM kernel's own tcgen05.mma kind::i8 shape (M = 128 * ctas,
- * N = 256, K = 32) back to back on operand tiles that stay in shared memory (pseudo-random bytes; no TMA, no
- * stores) for about `seconds` (0 < seconds <= 5; a short calibration launch sizes the timed launch).
- * Host outputs: *tops = 2 M N K * instructions / time in 1e12 op/s (required), *elapsed_ms and *sms_used
- * (either may be NULL).  `dev_status` (device int32, may be NULL) receives Q8_ERR_TIMEOUT bits should a wait
- * inside the kernel give up.  Synchronises `stream`.  Returns Q8_ERR_ARG on bad arguments, Q8_ERR_CUDA when a
- * runtime call fails. */
-q8_status q8_measure_int8_mma_peak(int ctas, double seconds, double *tops, double *elapsed_ms, int *sms_used,
-                                   void *dev_status, void *stream);
-
-/* Measurement aid, no counterpart in the paper: the one-directional HBM rates of the current device.  A copy
- * moves one byte in per byte out; the FC layers write 4 M N bytes of fp32 against M K + N K bytes of Int8
- * operands, so what bounds their output-heavy shapes is the store-only rate, which is well below the copy rate.
- * `buf` (device, 16-byte aligned, caller-owned, at least `bytes` long; make it several times the L2 size) is
- * overwritten with a pattern `repeats` times (store != 0) or read `repeats` times (store == 0) by a plain
- * grid-stride kernel of 16-byte accesses after one untimed pass.  Host outputs: *gbs = bytes * repeats / time in
- * 1e9 B/s (required), *elapsed_ms (may be NULL).  Synchronises `stream`.  Allocates no device memory.
- * Returns Q8_ERR_NULL / Q8_ERR_ALIGN / Q8_ERR_ARG (bytes < 16, repeats outside 1..1000) / Q8_ERR_CUDA. */
-q8_status q8_measure_hbm_peak(void *buf, size_t bytes, int store, int repeats, double *gbs, double *elapsed_ms,
-                              void *stream);
 
 #ifdef __cplusplus
 }

@@ -21,7 +21,7 @@ Q8_ERR_OVERFLOW, Q8_ERR_WORKSPACE, Q8_ERR_TIMEOUT, Q8_ERR_CUDA, Q8_ERR_ARG = 6, 
 Q8_ACT_NONE, Q8_ACT_GELU = 0, 1
 Q8_MAX_K = 133144
 
-# name -> (restype, argtypes); mirrors include/q8.h one to one.
+# name -> (restype, argtypes); mirrors include/q8.h and include/q8_tools.h one to one.
 _vp, _i64, _sz, _int, _f = C.c_void_p, C.c_int64, C.c_size_t, C.c_int, C.c_float
 SIGNATURES = {
     "q8_quantize_weight": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp]),
@@ -51,6 +51,7 @@ SIGNATURES = {
     "q8_tune_gemm_tile": (_int, [_int, _int]),
     "q8_tune_gemm_tail_split": (None, [_int]),
     "q8_tune_attention": (None, [_int]),
+    "q8_selftest_wait_timeout": (_int, [C.c_uint64, _vp, _vp, _vp]),
     "q8_attention_status_word": (_int, [C.POINTER(C.c_void_p)]),
     "q8_tune_gemm_epilogue_warps": (_int, [_int]),
     "q8_last_launch_tail_split": (_int, []),
@@ -454,6 +455,14 @@ def q8_measure_hbm_peak(buf: torch.Tensor, store: bool, repeats: int = 10, strea
                                     C.byref(ms), _stream(stream))
     _check(st, "q8_measure_hbm_peak")
     return {"gbs": gbs.value, "elapsed_ms": ms.value, "bytes": nbytes, "repeats": int(repeats), "store": bool(store)}
+
+
+def q8_selftest_wait_timeout(limit_ns: int, dev_status: torch.Tensor, dev_report: Optional[torch.Tensor] = None,
+                             stream=None) -> None:
+    """Launches the library's wait self-test: one CTA waits (bounded by limit_ns) on a barrier nobody arrives on."""
+    st = load().q8_selftest_wait_timeout(int(limit_ns), _ptr(dev_status, torch.int32, "dev_status"),
+                                         _ptr(dev_report, torch.int32, "dev_report"), _stream(stream))
+    _check(st, "q8_selftest_wait_timeout")
 
 
 def q8_tune_attention(use_tensor_cores: bool = True) -> None:

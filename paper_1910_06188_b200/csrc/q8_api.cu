@@ -39,7 +39,7 @@ q8_status quantize_tensor(const float *X, int64_t numel, const float *S_given, i
         li.launches += numel > 0 ? 2 : 1;
         S = S_dyn;
     }
-    Q8_CUDA_TRY(launch_quantize(X, numel, S, Xq, Xq_copy, s));
+    Q8_CUDA_TRY(launch_quantize(X, numel, S, Xq, Xq_copy, s, nullptr, S_given != nullptr ? status : nullptr));
     li.launches += numel > 0 ? 1 : 0;
     return Q8_OK;
 }
@@ -200,9 +200,10 @@ q8_status q8_calibrate(const float *X, int64_t numel, float decay, void *state, 
     if (!aligned_to(X, 4) || !aligned_to(state, 16)) return Q8_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     CalibState *st = static_cast<CalibState *>(state);
+    if (numel == 0) return Q8_OK;  // an empty batch is no observation of max|x|: the running state stays as it is
     Q8_CUDA_TRY(launch_absmax(X, numel, &st->scratch_bits, s));
     Q8_CUDA_TRY(launch_ema_update(st, decay, s));
-    last_launch_info().launches = numel > 0 ? 2 : 1;
+    last_launch_info().launches = 2;
     return Q8_OK;
 }
 

@@ -123,6 +123,12 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
         }
     } else {
         S = __ldg(S_ptr);
+        // a caller-supplied scale (an Eq. 4 result) that is zero, negative or not finite cannot quantise anything
+        // meaningful: the call still runs, and the condition is reported like a bad derived scale
+        if (blockIdx.x == 0 && threadIdx.x == 0 && (!(S > 0.0f) || isinf(S))) {
+            int32_t *word = status != nullptr ? status : clear_word;
+            if (word != nullptr) atomicOr(word, 1 << Q8_ERR_SCALE);
+        }
     }
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
@@ -173,8 +179,8 @@ __global__ void ema_update_kernel(CalibState *st, float decay)
     float m = __uint_as_float(st->scratch_bits);
     st->scratch_bits = 0u;
     float ema;
-    if (st->n_batches == 0) {
-        ema = m;
+    if (st->n_batches == 0 || decay == 0.0f) {
+        ema = m;  // first batch, or no history kept: exactly this batch's maximum (the dynamic scale of Sec. 4.1)
     } else {
         // ema += (1 - d) * (m - ema), each operation rounded separately (no fused multiply-add)
         float one_minus_d = __fsub_rn(1.0f, decay);
@@ -305,15 +311,15 @@ cudaError_t launch_scale_from_absmax(const uint32_t *bits, float *S, int32_t *st
 }
 
 cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy, cudaStream_t s,
-                            int32_t *clear_word)
+                            int32_t *clear_word, int32_t *status)
 {
     if (n <= 0) return cudaSuccess;
     if (aligned16(x) && aligned16(xq) && (xq_copy == nullptr || aligned16(xq_copy))) {
         return launch_overlapping_tail(quantize_kernel<true>, dim3(grid_for((n + 3) >> 2, kThreads * 4, 8)), dim3(kThreads), 0, s,
-                                       x, n, S, xq, xq_copy, nullptr, nullptr, nullptr, clear_word);
+                                       x, n, S, xq, xq_copy, nullptr, nullptr, status, clear_word);
     } else {
         quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, S, xq, xq_copy, nullptr, nullptr,
-                                                                                 nullptr, clear_word);
+                                                                                 status, clear_word);
     }
     return cudaGetLastError();
 }

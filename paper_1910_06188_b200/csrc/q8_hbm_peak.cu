@@ -5,7 +5,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "q8.h"
+#include "q8_tools.h"
 
 namespace q8 {
 namespace {

@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "q8.h"
+#include "q8_tools.h"
 
 namespace q8 {
 
@@ -60,8 +61,9 @@ cudaError_t launch_absmax(const float *x, int64_t n, uint32_t *bits, cudaStream_
 // *S = 127 / float(*bits) in place (bits and S may alias); flags Q8_ERR_SCALE on 0 / non-finite.
 cudaError_t launch_scale_from_absmax(const uint32_t *bits, float *S, int32_t *status, cudaStream_t s);
 // clear_word (may be NULL): a device word the kernel sets to zero before anything else (a call's status word).
+// A scale *S that is not a positive finite number raises Q8_ERR_SCALE in *status (or, without one, in *clear_word).
 cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *xq, int8_t *xq_copy,
-                            cudaStream_t s, int32_t *clear_word = nullptr);
+                            cudaStream_t s, int32_t *clear_word = nullptr, int32_t *status = nullptr);
 // Eq. 1 with S = 127 / float(*absmax_bits) derived inside the kernel (dynamic scale); *S_out receives S and
 // *status the Q8_ERR_SCALE bit when the maximum is 0 or not finite (S = 1 then).  absmax_bits and S_out differ.
 cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *absmax_bits, float *S_out,

@@ -8,6 +8,15 @@
 // that scratch in a fixed array that is part of the loaded library image on every GPU, so the call
 // itself allocates nothing.
 
+//
+// "Allocates nothing" describes the call itself once the library is warm on a device.  The first call on a
+// device (and the first call of each GEMM tile configuration) makes the CUDA runtime load the kernels and this
+// array onto that device and sets per-kernel attributes, which the runtime may serve with allocations of its
+// own; hosts with a frozen allocator should therefore issue one warm-up call per device and shape class during
+// initialisation.  The cached device addresses do not survive cudaDeviceReset.
+
+#include <atomic>
+
 #include "q8_internal.cuh"
 
 namespace {
@@ -20,18 +29,19 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 
 // In host code `g_static_scratch` is only a stand-in for the symbol; the device address has to be asked
 // for, once per device, with that device current.
-void *g_scratch_addr[64] = {};
+// Host threads may race to fill an entry; they all obtain the same address, so a plain atomic store suffices.
+std::atomic<void *> g_scratch_addr[64];
 
 q8_status static_scratch(void **out)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return Q8_ERR_CUDA;
-    if (g_scratch_addr[dev] == nullptr) {
-        void *p = nullptr;
+    void *p = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (p == nullptr) {
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return Q8_ERR_CUDA;
-        g_scratch_addr[dev] = p;
+        g_scratch_addr[dev].store(p, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = p;
     return Q8_OK;
 }
 

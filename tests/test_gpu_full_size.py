@@ -1,11 +1,10 @@
 """Parity at the benchmark's full size and launch configuration: the BERT-Large FC set at
 M = 24576 tokens with static scales, automatic tile choice (CTA pairs on 256 x 256 tiles).
 
-The oracle cannot run 0.6 tera-ops in seconds, so: the quantised activation is compared in full;
-three row slabs (first rows, rows straddling a tile boundary in the middle, last rows) are compared
-with the oracle on exactly those rows (rows are independent once the scale is fixed); random single
-entries are checked one by one; and the whole Int32 matrix is compared with the generic CUDA-core
-kernel as a secondary, on-device check."""
+The CPU oracle computes every one of the 24576 rows of each layer (a few seconds per layer on a
+multi-core host), so the whole quantised activation, the whole Int32 matrix and the whole fp32
+output are compared with it, element by element.  The generic CUDA-core kernel is compared as well,
+but only as a secondary, on-device cross-check: it is part of the same library, not a reference."""
 import numpy as np
 import pytest
 import torch
@@ -47,28 +46,20 @@ def test_bert_large_fc_full_size(name, K, N, act):
     assert q8.q8_poll_status(ws) == (q8.Q8_OK, 0)
     assert info["gemm_kernel"] == 1 and info["ctas"] == 2 and info["block_n"] == 256  # what bench.py times
 
-    # (1) the whole quantised activation
-    xq_ref = o.quantize(X, S_x)
-    assert np.array_equal(xq.cpu().numpy(), xq_ref)
+    # the oracle on all M rows: X_q, acc + b_q and Y, whole matrices
+    ref = o.linear(X, Wq_ref, S_w_ref, S_x, b, act)
+    assert ref["flags"] == 0
+    assert np.array_equal(xq.cpu().numpy(), ref["xq"]), f"{name}: X_q"
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"]), f"{name}: Int32 matrix"
+    Yh = Y.cpu().numpy()
+    scale = np.abs(ref["y"]).max()
+    worst = 0.0
+    for lo in range(0, M, 4096):   # in slabs, to keep the fp64 temporaries small
+        worst = max(worst, float(np.abs(Yh[lo:lo + 4096] - ref["y"][lo:lo + 4096]).max()))
+    assert worst <= REL_TOL * scale, f"{name}: max |Y - oracle| {worst:.3e} vs {REL_TOL} * {scale:.3e}"
+    del ref, Yh
 
-    # (2) row slabs against the oracle on the same rows
-    mid = (M // 2 // 256) * 256
-    for lo, hi in [(0, 48), (mid - 24, mid + 24), (M - 40, M)]:
-        ref = o.linear(X[lo:hi], Wq_ref, S_w_ref, S_x, b, act)
-        assert np.array_equal(acc[lo:hi].cpu().numpy(), ref["acc"]), f"{name}: Int32 rows {lo}:{hi}"
-        err = np.abs(Y[lo:hi].cpu().numpy().astype(np.float64) - ref["y"]).max()
-        assert err <= REL_TOL * np.abs(ref["y"]).max(), f"{name}: rows {lo}:{hi} err {err}"
-
-    # (3) random single entries, one by one
-    rng = np.random.default_rng(1234 + idx)
-    ms = rng.integers(0, M, size=200)
-    ns = rng.integers(0, N, size=200)
-    bq = o.quantize_bias(b, S_x, S_w_ref)
-    got = acc[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].cpu().numpy()
-    for m, n, g in zip(ms, ns, got):
-        assert o.linear_entry(xq_ref[m], Wq_ref[n], int(bq[n])) == g, f"{name}: entry ({m},{n})"
-
-    # (4) the whole Int32 matrix against the generic kernel (secondary, on-device)
+    # secondary, on-device: the generic kernel of this library gives the same Int32 matrix
     acc2 = torch.empty_like(acc)
     Y2 = q8.q8_linear_generic(Xd, Wq, S_w, S_x_dev, bd, act, workspace=ws, dbg_acc=acc2)
     assert q8.q8_last_launch_info()["gemm_kernel"] == 2
@@ -184,18 +175,30 @@ def test_int8_only_output_at_full_size():
     info = q8.q8_last_launch_info()
     assert q8.q8_poll_status(st) == (q8.Q8_OK, 0)
     assert (info["gemm_kernel"], info["block_n"], info["ctas"]) == (1, 256, 2)
-    # row slabs through the oracle's Eq. 1 (first rows, rows across a tile boundary in the middle, last rows)
-    mid = (M // 2 // 256) * 256
-    for lo, hi in [(0, 64), (mid - 40, mid + 40), (M - 300, M)]:
-        assert np.array_equal(Yq[lo:hi].cpu().numpy(), o.quantize(Y[lo:hi].cpu().numpy(), 37.5))
-    # the whole tensor against Eq. 1 in plain torch ops on the device (secondary: one rounded fp32 multiply,
-    # nearest-even integer, symmetric clamp)
+    # the fp32 output of the plain call against the oracle's steps on all rows (Int8 GEMM, Int32 bias, dequantise,
+    # GELU), then the Int8 output against the oracle's Eq. 1 applied to that fp32 output, everywhere
+    Wq_h, S_w_h = Wq.cpu().numpy(), S_w.item()
+    acc_ref, bad = o.gemm_s8(Xq.cpu().numpy(), Wq_h)
+    acc_ref, bad2 = o.add_bias(acc_ref, o.quantize_bias(bb.cpu().numpy(), 4.25, S_w_h))
+    assert bad == 0 and bad2 == 0
+    y_ref = o.gelu(o.dequantize(acc_ref, 4.25, S_w_h))
+    del acc_ref
+    Yh = Y.cpu().numpy()
+    assert np.abs(Yh - y_ref).max() <= REL_TOL * np.abs(y_ref).max()
+    Yq_h = Yq.cpu().numpy()
+    assert np.array_equal(Yq_h, o.quantize(Yh, 37.5))
+    # against the oracle's own fp64 output the Int8 value may differ by one step, and only where y * S_y sits
+    # within fp32 rounding of a tie
+    d = np.abs(Yq_h.astype(np.int16) - o.quantize(y_ref.astype(np.float32), 37.5).astype(np.int16))
+    assert d.max() <= 1 and (d != 0).mean() < 1e-3
+    del y_ref, Yh, Yq_h, d
+    # secondary, on the device: Eq. 1 in plain torch ops (one rounded fp32 multiply, nearest-even, symmetric clamp)
     assert torch.equal(Yq, torch.clamp(torch.round(Y * 37.5), -127, 127).to(torch.int8))
 
 
 def test_fused_qkv_with_per_layer_scales_at_full_size():
     """BERT-Large Q, K and V as one [3072, 1024] matrix with one Eq. 3 scale per 1024-row layer, M = 24576, in the
-    benchmark's launch configuration (CTA pairs): row slabs equal three separate oracle layers."""
+    benchmark's launch configuration (CTA pairs): the whole output equals three separate oracle layers."""
     H = 1024
     X = synth.activation(M, H, seed=1800)
     Ws = [synth.normal((H, H), 0.02 * (1 + i), 1801 + i) for i in range(3)]
@@ -206,15 +209,14 @@ def test_fused_qkv_with_per_layer_scales_at_full_size():
     Y = q8.q8_linear_wseg(dev(X), Wq, S_w, H, dev(np.array([S_x], np.float32)), dev(np.concatenate(bs)), 0, dbg_acc=acc)
     info = q8.q8_last_launch_info()
     assert (info["gemm_kernel"], info["block_n"], info["ctas"]) == (1, 256, 2)
-    mid = (M // 2 // 256) * 256
+    acc_h, Yh = acc.cpu().numpy(), Y.cpu().numpy()
     for i in range(3):
         Wq_ref, S_ref, _ = o.quantize_weight(Ws[i])
         assert S_w[i].item() == S_ref and np.array_equal(Wq[i * H:(i + 1) * H].cpu().numpy(), Wq_ref)
-        for lo, hi in [(0, 40), (mid - 20, mid + 20), (M - 40, M)]:
-            ref = o.linear(X[lo:hi], Wq_ref, S_ref, S_x, bs[i], 0)
-            assert np.array_equal(acc[lo:hi, i * H:(i + 1) * H].cpu().numpy(), ref["acc"]), (i, lo)
-            err = np.abs(Y[lo:hi, i * H:(i + 1) * H].cpu().numpy().astype(np.float64) - ref["y"]).max()
-            assert err <= REL_TOL * np.abs(ref["y"]).max(), (i, lo, err)
+        ref = o.linear(X, Wq_ref, S_ref, S_x, bs[i], 0)       # all M rows of this layer
+        assert np.array_equal(acc_h[:, i * H:(i + 1) * H], ref["acc"]), i
+        err = np.abs(Yh[:, i * H:(i + 1) * H] - ref["y"]).max()
+        assert err <= REL_TOL * np.abs(ref["y"]).max(), (i, err)
 
 
 def test_every_tile_shape_gives_the_same_bits():

@@ -88,11 +88,15 @@ def test_calibrate_decay_zero_is_dynamic_and_zero_batch_flags():
     for i, g in enumerate((3.0, 0.5, 7.0)):
         x = synth.activation(8, 40, seed=310 + i) * np.float32(g)
         q8.q8_calibrate(dev(x), 0.0, state)
-        ref.update(o.absmax(x), 0.0)
+        ref.update_batch(x, 0.0)
         got = state.view(torch.float32)[1].item()
-        assert np.float32(got) == ref.S_x                      # same fp32 steps as the oracle
-        # decay 0 tracks the last batch: ema + 1*(m - ema) is m up to one fp32 rounding
-        assert abs(got - 127.0 / float(o.absmax(x))) <= 4e-7 * got
+        # decay 0 keeps no history: exactly the dynamic scale of Sec. 4.1 for this batch
+        assert np.float32(got) == ref.S_x == np.float32(127.0) / o.absmax(x)
+    # an empty batch is no observation: state (ema, S_x, n_batches) unchanged, nothing launched
+    before = state.clone()
+    q8.q8_calibrate(torch.empty(0, device="cuda"), 0.5, state)
+    assert q8.q8_last_launch_info()["launches"] == 0 and torch.equal(state, before)
+    assert ref.update_batch(np.zeros(0, np.float32), 0.5) == np.float32(state.view(torch.float32)[1].item())
     state = q8.new_calibrate_state()
     q8.q8_calibrate(torch.zeros(100, device="cuda"), 0.9, state)
     assert state[4].item() == 1 << q8.Q8_ERR_SCALE and state.view(torch.float32)[1].item() == 1.0
@@ -187,6 +191,16 @@ def test_device_side_errors_are_returned_as_codes():
     ws = q8.new_workspace(8, 4, 16)
     Y = q8.q8_linear(X, Wq, S_w, None, None, 0, workspace=ws)      # max|X| == 0
     assert q8.q8_poll_status(ws)[0] == q8.Q8_ERR_SCALE and not Y.any()
+    # a caller-supplied static scale that is zero, negative, NaN or infinite is reported the same way
+    Xr = torch.randn((8, 16), device="cuda")
+    for bad in (0.0, -3.0, float("nan"), float("inf")):
+        q8.q8_linear(Xr, Wq, S_w, torch.full((1,), bad, device="cuda"), None, 0, workspace=ws)
+        assert q8.q8_poll_status(ws)[0] == q8.Q8_ERR_SCALE, bad
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        q8.q8_quantize_activation(Xr, torch.full((1,), bad, device="cuda"), dev_status=st)
+        assert q8.q8_poll_status(st)[0] == q8.Q8_ERR_SCALE, bad
+    q8.q8_linear(Xr, Wq, S_w, torch.full((1,), 2.5, device="cuda"), None, 0, workspace=ws)
+    assert q8.q8_poll_status(ws) == (q8.Q8_OK, 0)
     with pytest.raises(q8.Q8Error) as e:
         q8.q8_linear(X, Wq, S_w, None, None, 0, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.status == q8.Q8_ERR_WORKSPACE

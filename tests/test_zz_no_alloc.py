@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import q8_oracle as o
 from paper_1910_06188_b200 import binding as q8
 from paper_1910_06188_b200 import synth
 
@@ -22,6 +23,12 @@ def _case(M, N, K, act, seed, static_scale):
     b = _dev(synth.bias(N, seed + 2))
     S_x = torch.full((1,), 21.0, device="cuda") if static_scale else None
     return X, Wq, S_w, S_x, b, act
+
+
+def _oracle(X, Wq, S_w, S_x, b, act):
+    """The CPU oracle on the same inputs (the weight is the library's own Eq. 3 result, checked elsewhere)."""
+    return o.linear(X.cpu().numpy(), Wq.cpu().numpy(), S_w.item(), None if S_x is None else S_x.item(),
+                    b.cpu().numpy(), act)
 
 
 def test_noalloc_matches_q8_linear_on_two_calls_in_a_row():
@@ -43,6 +50,27 @@ def test_noalloc_matches_q8_linear_on_two_calls_in_a_row():
         assert (got - want).abs().max().item() <= tol
         want_xq, _ = q8.q8_quantize_activation(X, S_x)
         assert torch.equal(got_xq, want_xq)
+        # ... and against the CPU oracle: integers bit for bit, fp32 within 1e-5 of the output magnitude
+        ref = _oracle(X, Wq, S_w, S_x, b, act)
+        assert np.array_equal(got_xq.cpu().numpy(), ref["xq"]) and np.array_equal(got_acc.cpu().numpy(), ref["acc"])
+        assert np.abs(got.cpu().numpy() - ref["y"]).max() <= 1e-5 * np.abs(ref["y"]).max()
+
+
+def test_noalloc_call_leaves_device_memory_as_it_found_it():
+    """After a warm-up call, a call with caller-owned outputs takes no device memory: neither the driver's free
+    byte count nor torch's allocator statistics move across it."""
+    X, Wq, S_w, S_x, b, act = _case(512, 256, 384, 1, 2021, static_scale=True)
+    Y = torch.empty((512, 256), device="cuda")
+    q8.q8_linear_noalloc(X, Wq, S_w, S_x, b, act, Y=Y)      # warm-up: kernels and the scratch array get loaded
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    got, _ = q8.q8_linear_noalloc(X, Wq, S_w, S_x, b, act, Y=Y)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
+    ref = _oracle(X, Wq, S_w, S_x, b, act)
+    assert np.abs(got.cpu().numpy() - ref["y"]).max() <= 1e-5 * np.abs(ref["y"]).max()
 
 
 def test_noalloc_refuses_activations_beyond_its_fixed_scratch():
