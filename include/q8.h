@@ -210,6 +210,28 @@ q8_status q8_add_layernorm_quant(const float *x, const float *r1, const float *r
 q8_status q8_attention_quant(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx,
                              const float *S_q, int8_t *ctx_q, void *stream);
 
+/* Dynamic quantisation without stand-alone abs-max passes (Sec. 4.1: the scale 127 / max|x| is computed for every
+ * incoming activation tensor).  The kernel that PRODUCES an activation can fold max|y| of what it stores into a
+ * caller-owned device word while it writes it, and the quantised layer that consumes the activation takes its
+ * dynamic scale from that word instead of reading the whole tensor once more:
+ *   absmax_bits / y_absmax: device uint32 holding the IEEE bits of a non-negative fp32 (0 before the producer runs:
+ *     the caller clears it; producers only ever raise it, with an atomic max, so several producers may share a word
+ *     when their union is the tensor).  NaN outputs are skipped, an infinite output makes the word +Inf.
+ *   q8_add_layernorm_absmax / q8_attention_absmax: q8_add_layernorm / q8_attention plus that word.
+ *   q8_linear_dyn: q8_linear with the dynamic scale S_x = 127 / float(*x_absmax) (required; the word must be final,
+ *     i.e. its producer ordered before this call on the stream); S_x is left in the workspace header as in q8_linear,
+ *     Q8_ERR_SCALE is flagged there when the word is 0 or +Inf.  y_absmax (may be NULL) receives max|Y| of this
+ *     layer's own output (after GELU when act says so) for the next dynamically quantised layer.
+ * The results are bit-identical to q8_add_layernorm, q8_attention and q8_linear with S_x == NULL. */
+q8_status q8_add_layernorm_absmax(const float *x, const float *r1, const float *r2, const float *gamma,
+                                  const float *beta, float eps, int64_t rows, int64_t H, float *out,
+                                  uint32_t *absmax_bits, void *stream);
+q8_status q8_attention_absmax(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx,
+                              uint32_t *absmax_bits, void *stream);
+q8_status q8_linear_dyn(const float *X, const uint32_t *x_absmax, const int8_t *Wq, const float *S_w,
+                        const float *bias, int act, float *Y, uint32_t *y_absmax, int64_t M, int64_t N, int64_t K,
+                        void *workspace, size_t workspace_bytes, int8_t *dbg_Xq, int32_t *dbg_acc, void *stream);
+
 /* Synchronises `stream`, reads the device status word at `dev_status` (a q8_linear workspace
  * pointer works: the word sits at offset 0), clears it, and returns the lowest-numbered code
  * whose bit was set (Q8_OK if none).  `raw_bits` (host pointer, may be NULL) receives the word. */

@@ -38,6 +38,9 @@ SIGNATURES = {
     "q8_embedding": (_int, [_vp, _i64, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _vp]),
     "q8_add_layernorm": (_int, [_vp, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp]),
     "q8_attention": (_int, [_vp, _i64, _i64, _i64, _vp, _vp]),
+    "q8_add_layernorm_absmax": (_int, [_vp, _vp, _vp, _vp, _vp, _f, _i64, _i64, _vp, _vp, _vp]),
+    "q8_attention_absmax": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "q8_linear_dyn": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
     "q8_quantize_weight_segments": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "q8_linear_wseg": (_int, [_vp, _vp, _vp, _i64, _vp, _vp, _int, _vp, _i64, _i64, _i64, _vp, _sz, _vp, _vp, _vp]),
     "q8_linear_q_wseg": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _int, _vp, _i64, _i64, _i64, _vp, _vp, _vp]),
@@ -318,6 +321,56 @@ def q8_attention(qkv, B: int, S: int, heads: int, ctx=None, stream=None):
                              _stream(stream))
     _check(st, "q8_attention")
     return ctx
+
+
+def q8_add_layernorm_absmax(x, absmax_bits, r1=None, r2=None, gamma=None, beta=None, eps: float = 1e-12, out=None,
+                            stream=None):
+    """q8_add_layernorm that also folds max|out| into the int32 device word `absmax_bits` (fp32 bits; Sec. 4.1)."""
+    rows, H = x.shape
+    if out is None:
+        out = torch.empty_like(x)
+    st = load().q8_add_layernorm_absmax(_ptr(x, torch.float32, "x"), _ptr(r1, torch.float32, "r1"),
+                                        _ptr(r2, torch.float32, "r2"), _ptr(gamma, torch.float32, "gamma"),
+                                        _ptr(beta, torch.float32, "beta"), float(eps), rows, H,
+                                        _ptr(out, torch.float32, "out"), _ptr(absmax_bits, torch.int32, "absmax_bits"),
+                                        _stream(stream))
+    _check(st, "q8_add_layernorm_absmax")
+    return out
+
+
+def q8_attention_absmax(qkv, B: int, S: int, heads: int, absmax_bits, ctx=None, stream=None):
+    """q8_attention that also folds max|ctx| into the int32 device word `absmax_bits` (fp32 bits; Sec. 4.1)."""
+    H = heads * 64
+    if tuple(qkv.shape) != (B * S, 3 * H):
+        raise ValueError(f"qkv must be [{B * S}, {3 * H}], got {tuple(qkv.shape)}")
+    if ctx is None:
+        ctx = torch.empty((B * S, H), dtype=torch.float32, device=qkv.device)
+    st = load().q8_attention_absmax(_ptr(qkv, torch.float32, "qkv"), B, S, heads, _ptr(ctx, torch.float32, "ctx"),
+                                    _ptr(absmax_bits, torch.int32, "absmax_bits"), _stream(stream))
+    _check(st, "q8_attention_absmax")
+    return ctx
+
+
+def q8_linear_dyn(X, x_absmax, Wq, S_w, bias=None, act: int = Q8_ACT_NONE, Y=None, y_absmax=None, workspace=None,
+                  dbg_Xq=None, dbg_acc=None, stream=None) -> torch.Tensor:
+    """q8_linear with the dynamic scale 127 / max|X| taken from the device word `x_absmax` (written by the kernel
+    that produced X); `y_absmax` optionally receives max|Y| for the next dynamically quantised layer."""
+    M, K = X.shape
+    N, K2 = Wq.shape
+    if K != K2:
+        raise ValueError(f"X is [M,{K}] but Wq is [N,{K2}]")
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float32, device=X.device)
+    if workspace is None:
+        workspace = new_workspace(M, N, K, X.device)
+    st = load().q8_linear_dyn(_ptr(X, torch.float32, "X"), _ptr(x_absmax, torch.int32, "x_absmax"),
+                              _ptr(Wq, torch.int8, "Wq"), _ptr(S_w, torch.float32, "S_w"),
+                              _ptr(bias, torch.float32, "bias"), int(act), _ptr(Y, torch.float32, "Y"),
+                              _ptr(y_absmax, torch.int32, "y_absmax"), M, N, K, _any_ptr(workspace, "workspace"),
+                              workspace.numel() * workspace.element_size(), _ptr(dbg_Xq, torch.int8, "dbg_Xq"),
+                              _ptr(dbg_acc, torch.int32, "dbg_acc"), _stream(stream))
+    _check(st, "q8_linear_dyn")
+    return Y
 
 
 def q8_quantize_weight_segments(W, seg_rows: int, dev_status=None, stream=None):

@@ -69,7 +69,7 @@ q8_status run_gemm(const GemmArgs &g, bool force_generic, cudaStream_t s)
 q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
                       float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
                       int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic, int8_t *Yq,
-                      const float *S_y, int64_t w_seg)
+                      const float *S_y, int64_t w_seg, const uint32_t *x_absmax, uint32_t *y_absmax)
 {
     last_launch_info() = LaunchInfo();
     q8_status st = check_gemm_shape(M, N, K);
@@ -92,8 +92,14 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
     // Eq. 1.  With a given scale the quantise kernel itself starts the call's status word at zero (no separate
     // clearing operation in the stream); with the Sec. 4.1 dynamic scale (S_x NULL) the header is zeroed first, then
     // come the abs-max pass and one kernel that turns the maximum into the scale and quantises with it.
+    if ((x_absmax && !aligned_to(x_absmax, 4)) || (y_absmax && !aligned_to(y_absmax, 4))) return Q8_ERR_ALIGN;
     if (S_x != nullptr) {
         Q8_CUDA_TRY(launch_quantize(X, M * K, S_x, Xq, dbg_Xq, s, &hdr->status));
+        last_launch_info().launches += 1;
+    } else if (x_absmax != nullptr) {
+        // Sec. 4.1 with max|X| already known (folded into a device word by the kernel that produced X): one kernel
+        // derives the scale from it, publishes it in the header and quantises; it also starts the status word at zero.
+        Q8_CUDA_TRY(launch_quantize_dynamic(X, M * K, x_absmax, &hdr->S_x_dyn, &hdr->status, Xq, dbg_Xq, s, true));
         last_launch_info().launches += 1;
     } else {
         Q8_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), s));
@@ -113,6 +119,7 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
     g.Yq = Yq;
     g.S_y = S_y;
     g.dbg_acc = dbg_acc;
+    g.y_absmax = y_absmax;
     g.status = &hdr->status;
     g.M = M;
     g.N = N;
@@ -345,7 +352,7 @@ q8_status q8_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const fl
 
 static q8_status add_layernorm_impl(const float *x, const float *r1, const float *r2, const float *gamma,
                                     const float *beta, float eps, int64_t rows, int64_t H, float *out, const float *S_q,
-                                    int8_t *out_q, void *stream)
+                                    int8_t *out_q, void *stream, uint32_t *amax = nullptr)
 {
     last_launch_info() = LaunchInfo();
     if (rows < 0 || H < 0 || H > 12288 || rows > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
@@ -353,9 +360,9 @@ static q8_status add_layernorm_impl(const float *x, const float *r1, const float
     if (!x || (!out && !out_q) || (out_q && !S_q)) return Q8_ERR_NULL;
     if (!(eps >= 0.0f)) return Q8_ERR_ARG;
     if (!aligned_to(x, 4) || !aligned_to(out, 4) || !aligned_to(r1, 4) || !aligned_to(r2, 4) || !aligned_to(gamma, 4) ||
-        !aligned_to(beta, 4) || !aligned_to(S_q, 4))
+        !aligned_to(beta, 4) || !aligned_to(S_q, 4) || !aligned_to(amax, 4))
         return Q8_ERR_ALIGN;
-    Q8_CUDA_TRY(launch_add_layernorm(x, r1, r2, gamma, beta, eps, rows, H, out, S_q, out_q,
+    Q8_CUDA_TRY(launch_add_layernorm(x, r1, r2, gamma, beta, eps, rows, H, out, S_q, out_q, amax,
                                      static_cast<cudaStream_t>(stream)));
     last_launch_info().launches = 1;
     return Q8_OK;
@@ -377,14 +384,15 @@ q8_status q8_add_layernorm_quant(const float *x, const float *r1, const float *r
 }
 
 static q8_status attention_impl(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
-                                int8_t *ctx_q, void *stream)
+                                int8_t *ctx_q, void *stream, uint32_t *amax = nullptr)
 {
     last_launch_info() = LaunchInfo();
     if (B < 0 || S < 0 || heads < 0 || B > 65535 || heads > 65535 || S > (int64_t)INT_MAX) return Q8_ERR_SHAPE;
     if (B == 0 || S == 0 || heads == 0) return Q8_OK;
     if (!qkv || (!ctx && !ctx_q) || (ctx_q && !S_q)) return Q8_ERR_NULL;
-    if (!aligned_to(qkv, 8) || !aligned_to(ctx, 8) || !aligned_to(S_q, 4)) return Q8_ERR_ALIGN;  // 8-byte vector accesses
-    Q8_CUDA_TRY(launch_attention(qkv, B, S, heads, ctx, S_q, ctx_q, static_cast<cudaStream_t>(stream)));
+    if (!aligned_to(qkv, 8) || !aligned_to(ctx, 8) || !aligned_to(S_q, 4) || !aligned_to(amax, 4))
+        return Q8_ERR_ALIGN;  // 8-byte vector accesses
+    Q8_CUDA_TRY(launch_attention(qkv, B, S, heads, ctx, S_q, ctx_q, amax, static_cast<cudaStream_t>(stream)));
     last_launch_info().launches = 1;
     return Q8_OK;
 }
@@ -400,6 +408,30 @@ q8_status q8_attention_quant(const float *qkv, int64_t B, int64_t S, int64_t hea
 {
     if (B > 0 && S > 0 && heads > 0 && !ctx_q) return Q8_ERR_NULL;
     return attention_impl(qkv, B, S, heads, ctx, S_q, ctx_q, stream);
+}
+
+q8_status q8_add_layernorm_absmax(const float *x, const float *r1, const float *r2, const float *gamma,
+                                  const float *beta, float eps, int64_t rows, int64_t H, float *out,
+                                  uint32_t *absmax_bits, void *stream)
+{
+    if (!absmax_bits || (rows > 0 && H > 0 && !out)) return Q8_ERR_NULL;
+    return add_layernorm_impl(x, r1, r2, gamma, beta, eps, rows, H, out, nullptr, nullptr, stream, absmax_bits);
+}
+
+q8_status q8_attention_absmax(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, uint32_t *absmax_bits,
+                              void *stream)
+{
+    if (!absmax_bits || (B > 0 && S > 0 && heads > 0 && !ctx)) return Q8_ERR_NULL;
+    return attention_impl(qkv, B, S, heads, ctx, nullptr, nullptr, stream, absmax_bits);
+}
+
+q8_status q8_linear_dyn(const float *X, const uint32_t *x_absmax, const int8_t *Wq, const float *S_w, const float *bias,
+                        int act, float *Y, uint32_t *y_absmax, int64_t M, int64_t N, int64_t K, void *workspace,
+                        size_t workspace_bytes, int8_t *dbg_Xq, int32_t *dbg_acc, void *stream)
+{
+    if (M > 0 && N > 0 && (!Y || !x_absmax)) return Q8_ERR_NULL;
+    return linear_impl(X, Wq, S_w, nullptr, bias, act, Y, M, N, K, workspace, workspace_bytes, dbg_Xq, dbg_acc, stream,
+                       false, nullptr, nullptr, 0, x_absmax, y_absmax);
 }
 
 q8_status q8_poll_status(void *dev_status, uint32_t *raw_bits, void *stream)

@@ -88,7 +88,8 @@ __device__ __forceinline__ void worker_barrier() { asm volatile("bar.sync 1, %0;
 
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale, float *__restrict__ ctx,
-                    const float *__restrict__ S_q, int8_t *__restrict__ ctx_q, uint32_t tmem_cols, int32_t *status)
+                    const float *__restrict__ S_q, int8_t *__restrict__ ctx_q, uint32_t *__restrict__ amax,
+                    uint32_t tmem_cols, int32_t *status)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -334,6 +335,14 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             float y[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) y[j] = (__uint_as_float(v[j]) + __uint_as_float(w[j])) * inv;
+            if (amax != nullptr) {  // max|ctx| for a dynamically quantised consumer (Sec. 4.1); rows past S do not count
+                float am = 0.0f;
+                if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) am = fmaxf(am, fabsf(y[j]));
+                }
+                warp_fold_absmax(am, amax);
+            }
             if (ctx != nullptr && row_ok) {
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
@@ -388,7 +397,7 @@ bool attention_tc_supported(const float *qkv, int64_t S, int64_t heads, const fl
 }
 
 cudaError_t launch_attention_tc(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
-                                int8_t *ctx_q, cudaStream_t s)
+                                int8_t *ctx_q, uint32_t *amax, cudaStream_t s)
 {
     static bool attr_set[64] = {};
     int dev = 0;
@@ -406,7 +415,7 @@ cudaError_t launch_attention_tc(const float *qkv, int64_t B, int64_t S, int64_t 
     dim3 grid((unsigned)((S + kQTile - 1) / kQTile), (unsigned)heads, (unsigned)B);
     const float scale = 1.4426950408889634f / 8.0f;  // log2(e) / sqrt(64): the softmax then uses 2^x
     return launch_overlapping_tail(attention_tc_kernel, grid, dim3(kThreads), kAttnTcSmemBytes, s, qkv, (int)S,
-                                   heads * kHeadDim, scale, ctx, S_q, ctx_q, cols, attention_status_word());
+                                   heads * kHeadDim, scale, ctx, S_q, ctx_q, amax, cols, attention_status_word());
 }
 
 }  // namespace q8

@@ -325,15 +325,16 @@ cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *x
 }
 
 cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *absmax_bits, float *S_out, int32_t *status,
-                                    int8_t *xq, int8_t *xq_copy, cudaStream_t s)
+                                    int8_t *xq, int8_t *xq_copy, cudaStream_t s, bool clear_status)
 {
     if (n <= 0) return cudaSuccess;
+    int32_t *clear_word = clear_status ? status : nullptr;
     if (aligned16(x) && aligned16(xq) && (xq_copy == nullptr || aligned16(xq_copy))) {
         return launch_overlapping_tail(quantize_kernel<true>, dim3(grid_for((n + 3) >> 2, kThreads * 4, 8)), dim3(kThreads), 0, s,
-                                       x, n, nullptr, xq, xq_copy, absmax_bits, S_out, status, nullptr);
+                                       x, n, nullptr, xq, xq_copy, absmax_bits, S_out, status, clear_word);
     } else {
         quantize_kernel<false><<<grid_for(n, kThreads * 4, 8), kThreads, 0, s>>>(x, n, nullptr, xq, xq_copy, absmax_bits,
-                                                                                 S_out, status);
+                                                                                 S_out, status, clear_word);
     }
     return cudaGetLastError();
 }

@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(GemmArgs a)
 
     const float S_x = __ldg(a.S_x);
     const float S_y = a.Yq ? __ldg(a.S_y) : 1.0f;
+    float am = 0.0f;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int64_t n = n0 + tx * 4 + j;
@@ -64,10 +65,12 @@ __global__ void __launch_bounds__(256) gemm_generic_kernel(GemmArgs a)
             const int32_t v = add_wrap(acc[i][j], bq);
             if (a.dbg_acc) a.dbg_acc[m * a.N + n] = v;
             const float y = finish_output(v, inv, a.act);
+            am = fmaxf(am, fabsf(y));
             if (a.Y) a.Y[m * a.N + n] = y;
             if (a.Yq) a.Yq[m * a.N + n] = (int8_t)quantize_value(y, S_y);
         }
     }
+    if (a.y_absmax) warp_fold_absmax(am, a.y_absmax);
 }
 
 }  // namespace

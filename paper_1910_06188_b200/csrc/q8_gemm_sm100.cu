@@ -22,29 +22,33 @@
 
 #include <cuda.h>
 
-#include "q8_internal.cuh"
-#include "q8_sm100_ptx.cuh"
+#include "q8_gemm_common.cuh"
 
 namespace q8 {
 
 namespace {
 
 using namespace ptx;
+using namespace gemm_detail;
 
-constexpr int BLOCK_M = 128;       // accumulator rows per CTA: row i <-> TMEM lane i
-constexpr int BLOCK_K = 128;       // bytes == int8 elements per stage row: one 128-byte swizzle span
-constexpr int UMMA_K = 32;         // K of one kind::i8 instruction
 constexpr int kAccStages = 2;      // TMEM accumulator double buffering
 // Epilogue warps per CTA (template parameter EW): 8 = two per TMEM lane quarter, each taking half of the tile's
 // columns; 16 = four per quarter.  A warp walks its 32-column blocks one after the other and every block is a
 // chain of dependent latencies (TMEM load, arithmetic, staging, proxy fence, TMA store), so when the main loop is
 // short (small K) more warps shorten the epilogue; the extra staging buffers cost one stage of the operand ring.
-constexpr int kStagingBytesPerWarp = 32 * 32 * 4;  // the 32 x 32 fp32 block one tcgen05.ld hands to a warp
 
 template <int BLOCK_N, int CTAS, int EW>
 struct Cfg {
     static constexpr int kEpilogueWarps = EW;
-    static constexpr int kThreads = 64 + 32 * EW;
+    // With 16 epilogue warps the roles are aligned to warpgroups (warps 0..3: producer, MMA issuer, two idle warps;
+    // warps 4..19: epilogue) so that setmaxnreg can move registers from the issuing warpgroup to the epilogue warps:
+    // these then hold their whole 32 x 64 accumulator share at once and hand the TMEM buffer back before any arithmetic.
+    static constexpr bool kRegSplit = EW == 16;
+    static constexpr int kFirstEpilogueWarp = kRegSplit ? 4 : 2;
+    static constexpr int kThreads = 32 * (kFirstEpilogueWarp + EW);
+    static constexpr int kRegsIssue = 32, kRegsEpilogue = 112, kRegsAtLaunch = 96;
+    static_assert(!kRegSplit || 128 * kRegsIssue + 32 * EW * kRegsEpilogue <= kThreads * kRegsAtLaunch,
+                  "setmaxnreg split exceeds the registers of the launch");
     static constexpr int kBRows = BLOCK_N / CTAS;  // W_q rows each CTA loads
     static constexpr int kABytes = BLOCK_M * BLOCK_K;
     static constexpr int kBBytes = kBRows * BLOCK_K;
@@ -69,180 +73,9 @@ struct Cfg {
                                            | ((uint32_t)((BLOCK_M * CTAS) >> 4) << 24); // M / 16
 };
 
-// ---- GELU without erff, two values at a time: gelu(y) = max(y, 0) - a * Phi(-a), a = |y|, with
-// Phi(-a) = 2^p(a) and p a degree-6 fit of log2 Phi(-a) on [0, 5.6] (p(0) = -1 exactly; beyond 5.6
-// a * Phi(-a) < 1e-7 and a is clamped).  Absolute error of a * Phi(-a) below 1e-7, so the result is
-// within fp32 rounding of the erf form.  The polynomial runs on packed fp32 FMAs (two values per
-// instruction, each half rounded like a scalar fmaf) in n = -a = max(-|y|, -5.6), i.e. with the odd
-// coefficients negated, so the last step needs no negation: gelu = n * 2^p + max(y, 0).
-// Per value: three packed FMA-pipe instructions and a half, one ex2, two min/max.
-__device__ __forceinline__ void gelu_fast_x2(uint64_t y2, float &out_lo, float &out_hi)
-{
-    float y0, y1;
-    unpack_f32x2(y2, y0, y1);
-    const uint64_t n = pack_f32x2(fmaxf(-fabsf(y0), -5.6f), fmaxf(-fabsf(y1), -5.6f));
-    uint64_t p = pack_f32x2(2.9923698093625717e-05f, 2.9923698093625717e-05f);
-    p = fma_f32x2(p, n, pack_f32x2(0.0007398707093670964f, 0.0007398707093670964f));
-    p = fma_f32x2(p, n, pack_f32x2(0.007977453991770744f, 0.007977453991770744f));
-    p = fma_f32x2(p, n, pack_f32x2(0.05323817580938339f, 0.05323817580938339f));
-    p = fma_f32x2(p, n, pack_f32x2(-0.45891568064689636f, -0.45891568064689636f));
-    p = fma_f32x2(p, n, pack_f32x2(1.1511471271514893f, 1.1511471271514893f));
-    p = fma_f32x2(p, n, pack_f32x2(-1.0f, -1.0f));
-    float p0, p1, e0, e1;
-    unpack_f32x2(p, p0, p1);
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(p0));
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(p1));
-    const uint64_t r = fma_f32x2(n, pack_f32x2(e0, e1), pack_f32x2(fmaxf(y0, 0.0f), fmaxf(y1, 0.0f)));
-    unpack_f32x2(r, out_lo, out_hi);
-}
-
-// ------------------------------------------------------------------ epilogue of one warp
-// The warp owns 32 accumulator rows (its TMEM lane quarter) x COLS columns of the tile and walks
-// them in 32-column blocks: tcgen05.ld (one row per lane) -> + b_q -> int-to-float ->
-// * 1/(S_x S_w) -> GELU -> store.  With tma_store (N % 4 == 0, Y 16-byte aligned) the 32 x 32 fp32
-// block is staged in shared memory in the 128-byte-swizzled layout of the output tensor map
-// (row = lane, 16-byte piece g at position g ^ (lane & 7): bank-conflict free) and written by one
-// TMA store, clipped at the matrix edge by the hardware; otherwise every lane stores its own row.
-// Once the last TMEM load of the tile has landed the accumulator buffer is handed back (release()).
-template <int COLS, typename Release>
-__device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
-                                              const CUtensorMap *tmap_yq, bool yq_tma, uint32_t taddr, int64_t row0,
-                                              int64_t col0, const int32_t (&bqv)[COLS / 32], const float (&invv)[COLS / 32],
-                                              uint8_t *stage, int32_t *bq_s, int lane, int nch, Release release)
-{
-    constexpr int NCHUNK = COLS / 32;  // compile-time maximum; this tile has nch <= NCHUNK blocks (warp-uniform)
-    const int64_t row = row0 + lane;
-    const bool row_ok = row < a.M;
-    const float S_y = a.Yq != nullptr ? __ldg(a.S_y) : 1.0f;
-    const bool yq_vec = ((a.N & 15) == 0) && ((reinterpret_cast<uintptr_t>(a.Yq) & 15u) == 0);
-    // Int8-only output of a full-width tile: the warp's 32 x COLS bytes are collected in its staging buffer (free,
-    // since no fp32 block is staged) in the swizzled layout of the Int8 output tensor map and leave as one TMA
-    // store of whole 64- or 128-byte row pieces instead of 32 separate 16-byte stores per lane and block.
-    constexpr bool kYqStageable = COLS == 64 || COLS == 128;
-    const bool yq_staged = kYqStageable && yq_tma && nch == NCHUNK;
-    const int yq_xor = COLS == 128 ? (lane & 7) : ((lane >> 1) & 3);  // 128-byte / 64-byte swizzle of row `lane`
-    bool yq_pending = false;
-
-    // everything after the TMEM load, for the 32-column block ci held in v
-    auto finish_block = [&](uint32_t (&v)[32], int ci) {
-        const int64_t nb = col0 + 32 * ci;
-        const float inv = invv[ci];
-        if (nb >= a.N || row0 >= a.M) return;  // warp-uniform: the block lies outside the matrix
-        // b_q of these 32 columns (one per lane, computed before the accumulator was ready) -> all lanes
-        __syncwarp();
-        bq_s[lane] = bqv[ci];
-        __syncwarp();
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            const int4 b = *reinterpret_cast<const int4 *>(bq_s + 4 * g);
-            v[4 * g + 0] = (uint32_t)add_wrap((int32_t)v[4 * g + 0], b.x);
-            v[4 * g + 1] = (uint32_t)add_wrap((int32_t)v[4 * g + 1], b.y);
-            v[4 * g + 2] = (uint32_t)add_wrap((int32_t)v[4 * g + 2], b.z);
-            v[4 * g + 3] = (uint32_t)add_wrap((int32_t)v[4 * g + 3], b.w);
-        }
-        if (a.dbg_acc != nullptr && row_ok) {
-            int32_t *drow = a.dbg_acc + row * a.N + nb;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (nb + j < a.N) drow[j] = (int32_t)v[j];
-        }
-        if (a.act == Q8_ACT_GELU) {
-            const uint64_t inv2 = pack_f32x2(inv, inv);
-#pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-                const uint64_t y2 =
-                    mul_f32x2(pack_f32x2(__int2float_rn((int32_t)v[j]), __int2float_rn((int32_t)v[j + 1])), inv2);
-                float g0, g1;
-                gelu_fast_x2(y2, g0, g1);
-                v[j] = __float_as_uint(g0);
-                v[j + 1] = __float_as_uint(g1);
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__fmul_rn(__int2float_rn((int32_t)v[j]), inv));
-        }
-        if (a.Yq != nullptr && row_ok) {
-            // re-quantised output for the next quantised layer: Eq. 1 at that layer's activation scale
-            int8_t *qrow = a.Yq + row * a.N + nb;
-            if (yq_staged) {
-                // handled below, for all rows of the warp (rows past M are clipped by the store)
-            } else if (yq_vec) {  // N % 16 == 0: a 16-byte piece is never split by the edge
-                if (nb < a.N)
-                    *reinterpret_cast<uint4 *>(qrow) = make_uint4(
-                        quantize_pack4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]), S_y),
-                        quantize_pack4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]), S_y),
-                        quantize_pack4(__uint_as_float(v[8]), __uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]), S_y),
-                        quantize_pack4(__uint_as_float(v[12]), __uint_as_float(v[13]), __uint_as_float(v[14]), __uint_as_float(v[15]), S_y));
-                if (nb + 16 < a.N)
-                    *reinterpret_cast<uint4 *>(qrow + 16) = make_uint4(
-                        quantize_pack4(__uint_as_float(v[16]), __uint_as_float(v[17]), __uint_as_float(v[18]), __uint_as_float(v[19]), S_y),
-                        quantize_pack4(__uint_as_float(v[20]), __uint_as_float(v[21]), __uint_as_float(v[22]), __uint_as_float(v[23]), S_y),
-                        quantize_pack4(__uint_as_float(v[24]), __uint_as_float(v[25]), __uint_as_float(v[26]), __uint_as_float(v[27]), S_y),
-                        quantize_pack4(__uint_as_float(v[28]), __uint_as_float(v[29]), __uint_as_float(v[30]), __uint_as_float(v[31]), S_y));
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (nb + j < a.N) qrow[j] = (int8_t)quantize_value(__uint_as_float(v[j]), S_y);
-            }
-        }
-        if (yq_staged) {
-            if (!yq_pending) {
-                if (lane == 0) tma_store_wait_read();  // the previous tile has left the staging buffer
-                __syncwarp();
-                yq_pending = true;
-            }
-            uint8_t *srow = stage + lane * COLS;
-            *reinterpret_cast<uint4 *>(srow + (((2 * ci) ^ yq_xor) << 4)) = make_uint4(
-                quantize_pack4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]), S_y),
-                quantize_pack4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]), S_y),
-                quantize_pack4(__uint_as_float(v[8]), __uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]), S_y),
-                quantize_pack4(__uint_as_float(v[12]), __uint_as_float(v[13]), __uint_as_float(v[14]), __uint_as_float(v[15]), S_y));
-            *reinterpret_cast<uint4 *>(srow + (((2 * ci + 1) ^ yq_xor) << 4)) = make_uint4(
-                quantize_pack4(__uint_as_float(v[16]), __uint_as_float(v[17]), __uint_as_float(v[18]), __uint_as_float(v[19]), S_y),
-                quantize_pack4(__uint_as_float(v[20]), __uint_as_float(v[21]), __uint_as_float(v[22]), __uint_as_float(v[23]), S_y),
-                quantize_pack4(__uint_as_float(v[24]), __uint_as_float(v[25]), __uint_as_float(v[26]), __uint_as_float(v[27]), S_y),
-                quantize_pack4(__uint_as_float(v[28]), __uint_as_float(v[29]), __uint_as_float(v[30]), __uint_as_float(v[31]), S_y));
-        }
-        if (a.Y == nullptr) return;
-        if (tma_store) {
-            if (lane == 0) tma_store_wait_read();  // the previous block has left the staging buffer
-            __syncwarp();
-            uint8_t *srow = stage + lane * 128;
-#pragma unroll
-            for (int g = 0; g < 8; ++g)
-                *reinterpret_cast<uint4 *>(srow + ((g ^ (lane & 7)) << 4)) =
-                    make_uint4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-            fence_proxy_async_smem();  // generic-proxy writes above -> visible to the TMA (async proxy)
-            __syncwarp();
-            if (lane == 0) tma_store_2d(tmap_y, (int32_t)nb, (int32_t)row0, smem_u32(stage));
-        } else if (row_ok) {
-            float *yrow = a.Y + row * a.N + nb;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (nb + j < a.N) yrow[j] = __uint_as_float(v[j]);
-        }
-    };
-
-#pragma unroll
-    for (int ci = 0; ci < NCHUNK; ++ci) {
-        if (ci >= nch) break;
-        uint32_t v[32];
-        tmem_ld_32x32(taddr + (uint32_t)(32 * ci), v);
-        tmem_ld_wait();
-        if (ci + 1 == nch) release();
-        finish_block(v, ci);
-    }
-    if (yq_pending) {
-        // blocks beyond column N were never staged; the store clips them (and rows past M) at the matrix edge
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) tma_store_2d(tmap_yq, (int32_t)col0, (int32_t)row0, smem_u32(stage));
-    }
-}
-
 // ------------------------------------------------------------------ the kernel
 template <int BLOCK_N, int CTAS, int EW>
-__global__ void __launch_bounds__(64 + 32 * EW, 1)
+__global__ void __launch_bounds__(Cfg<BLOCK_N, CTAS, EW>::kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_w4,
                     const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_yq, GemmArgs a,
@@ -316,6 +149,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // produced X_q) must be complete before anything below reads global memory
     grid_dependency_wait();
 
+    // Each role's code sits in the same branch as its register-count change, so that it is compiled for that count.
+    if (warp < C::kFirstEpilogueWarp) {
+    if (C::kRegSplit) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsIssue));
     if (warp == 0) {
         // ---------------- TMA producer (each CTA loads its own rows) ----------------
         if (lane == 0) {
@@ -419,9 +255,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                        global_timer_ns() - t0 < 50000000ull) {}
             }
         }
+    }
     } else {
         // ---------------- epilogue ----------------
-        const int ew = warp - 2;       // 0 .. 7
+        if (C::kRegSplit) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsEpilogue));
+        const int ew = warp - C::kFirstEpilogueWarp;  // 0 .. EW-1
         const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32*quarter .. +31
         const int col_group = ew >> 2;  // which share of the tile's columns this warp takes
         const float S_x = __ldg(a.S_x);
@@ -436,6 +274,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         int as = 0;
         uint32_t aphase = 0;
         bool ok = true;
+        float absmax_run = 0.0f;  // max|y| over everything this lane has stored (only kept when a.y_absmax is given)
         // The bias values of a tile are fetched one tile ahead: under the operand traffic of the main loop a
         // global load takes microseconds, which would otherwise be exposed at the start of every tile.
         constexpr int NCH = C::kColsPerWarp / 32;
@@ -487,13 +326,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
             };
             if (active)
-                epilogue_warp<C::kColsPerWarp>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
+                epilogue_warp<C::kColsPerWarp, C::kRegSplit>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
-                                               m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release);
+                                               m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release,
+                                               absmax_run);
             else
                 release();
             if (++as == kAccStages) { as = 0; aphase ^= 1u; }
         }
+        if (a.y_absmax != nullptr) warp_fold_absmax(absmax_run, a.y_absmax);  // one atomic per epilogue warp and launch
         if (lane == 0) tma_store_wait_all();
     }
 
@@ -513,122 +354,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 }
 
 // ------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn()
-{
-    static EncodeTiledFn fn = [] {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// A tensor map depends only on the base address, the extents and the box, and a serving loop calls with the same
-// few buffers over and over, so the encoded maps are kept in a small per-thread table (direct-mapped on a hash of
-// those fields): a hit saves the driver call, which matters for launch-bound small problems.
-struct TmapKey {
-    const void *base;
-    int64_t d0, d1;
-    int32_t box0, box1, kind;
-    bool operator==(const TmapKey &o) const
-    {
-        return base == o.base && d0 == o.d0 && d1 == o.d1 && box0 == o.box0 && box1 == o.box1 && kind == o.kind;
-    }
-};
-struct TmapSlot {
-    TmapKey key;
-    CUtensorMap map;
-    bool valid = false;
-};
-constexpr int kTmapSlots = 64;
-
-template <typename Encode>
-bool cached_tmap(CUtensorMap *out, const TmapKey &key, Encode encode)
-{
-    static thread_local TmapSlot table[kTmapSlots];
-    uint64_t h = reinterpret_cast<uintptr_t>(key.base) * 0x9E3779B97F4A7C15ull;
-    h ^= (uint64_t)key.d0 * 0xC2B2AE3D27D4EB4Full + (uint64_t)key.d1 * 0x165667B19E3779F9ull +
-         (uint64_t)(key.box1 * 131 + key.box0 * 7 + key.kind);
-    TmapSlot &slot = table[(h >> 40) % kTmapSlots];
-    if (slot.valid && slot.key == key) {
-        *out = slot.map;
-        return true;
-    }
-    if (!encode(out)) return false;
-    slot.key = key;
-    slot.map = *out;
-    slot.valid = true;
-    return true;
-}
-
-// Row-major int8 matrix [rows, K] as a 2-D tensor map with (128 x box_rows) boxes, 128-byte swizzle.
-// Elements outside the matrix read as zero, which is what ragged M, N and K tails need.
-bool make_tmap(CUtensorMap *map, const int8_t *base, int64_t rows, int64_t K, int box_rows)
-{
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    return cached_tmap(map, TmapKey{base, K, rows, BLOCK_K, box_rows, 0}, [&](CUtensorMap *m) {
-        cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-        cuuint64_t strides[1] = {(cuuint64_t)K};
-        cuuint32_t box[2] = {(cuuint32_t)BLOCK_K, (cuuint32_t)box_rows};
-        cuuint32_t estr[2] = {1, 1};
-        return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-    });
-}
-
-// Row-major fp32 output [M, N] as a tensor map of 32 x 32 boxes (128 bytes wide), 128-byte swizzle.
-// Stores that reach past row M or column N are clipped by the hardware.
-bool make_tmap_out(CUtensorMap *map, float *base, int64_t M, int64_t N)
-{
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    return cached_tmap(map, TmapKey{base, N, M, 32, 32, 1}, [&](CUtensorMap *m) {
-        cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-        cuuint64_t strides[1] = {(cuuint64_t)N * 4};
-        cuuint32_t box[2] = {32, 32};
-        cuuint32_t estr[2] = {1, 1};
-        return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-    });
-}
-
-// Row-major Int8 output [M, N] as a tensor map of (box_cols x 32) boxes: 64-byte rows with the 64-byte swizzle
-// or 128-byte rows with the 128-byte swizzle.
-bool make_tmap_out_q(CUtensorMap *map, int8_t *base, int64_t M, int64_t N, int box_cols)
-{
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    return cached_tmap(map, TmapKey{base, N, M, box_cols, 32, 2}, [&](CUtensorMap *m) {
-        cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-        cuuint64_t strides[1] = {(cuuint64_t)N};
-        cuuint32_t box[2] = {(cuuint32_t)box_cols, 32};
-        cuuint32_t estr[2] = {1, 1};
-        return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  box_cols == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-    });
-}
-
-int sm_count()
-{
-    static int n = [] {
-        int dev = 0, v = 148;
-        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-        return v > 0 ? v : 148;
-    }();
-    return n;
-}
-
 int g_force_block_n = 0, g_force_ctas = 0;  // set by q8_tune_gemm_tile(); 0 = choose automatically
 int g_force_epilogue_warps = 0;            // 0 automatic, else 8 or 16 (cta_group::2 kernel only)
 bool g_tail_split_enabled = true;          // cut the tiles of a partial last round into narrower ones
@@ -646,6 +371,14 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
+        if (C::kRegSplit) {
+            // setmaxnreg.inc draws on the registers the block was launched with; a launch with fewer registers per
+            // thread than the split assumes would wait forever, so refuse it here
+            cudaFuncAttributes fa;
+            e = cudaFuncGetAttributes(&fa, kernel);
+            if (e != cudaSuccess) return e;
+            if (fa.numRegs < C::kRegsAtLaunch) return cudaErrorLaunchOutOfResources;
+        }
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         int units = sm_count() / CTAS;

@@ -39,6 +39,7 @@ struct GemmArgs {
     int8_t *Yq;         // [M,N] Int8 output Quantize(y | S_y) (Eq. 1 at the consumer's scale), or nullptr
     const float *S_y;   // device scalar, required with Yq
     int32_t *dbg_acc;   // [M,N] or nullptr
+    uint32_t *y_absmax = nullptr;  // optional: max|y| over the stored output is folded into this word (float bits, atomicMax)
     int32_t *status;    // device status word or nullptr
     int64_t M, N, K;
     int act;
@@ -66,24 +67,28 @@ cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *x
                             cudaStream_t s, int32_t *clear_word = nullptr, int32_t *status = nullptr);
 // Eq. 1 with S = 127 / float(*absmax_bits) derived inside the kernel (dynamic scale); *S_out receives S and
 // *status the Q8_ERR_SCALE bit when the maximum is 0 or not finite (S = 1 then).  absmax_bits and S_out differ.
+// clear_status: start *status at zero first (the call's status word, when no memset precedes the kernel).
 cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *absmax_bits, float *S_out,
-                                    int32_t *status, int8_t *xq, int8_t *xq_copy, cudaStream_t s);
+                                    int32_t *status, int8_t *xq, int8_t *xq_copy, cudaStream_t s,
+                                    bool clear_status = false);
 cudaError_t launch_ema_update(CalibState *st, float decay, cudaStream_t s);
 cudaError_t launch_fake_quantize(const float *x, int64_t n, const float *S, float *xhat, cudaStream_t s);
 cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,
                              int64_t H, float *out, int8_t *rows_q, int32_t *status, cudaStream_t s);
 
 // ---- fp32 encoder support (q8_support.cu) ----
+// amax (may be NULL): max|output| is folded into this device word (float bits, atomicMax; it must hold 0 or an
+// earlier maximum), so that a dynamically quantised consumer (Sec. 4.1) needs no abs-max pass of its own.
 cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma,
                                  const float *beta, float eps, int64_t rows, int64_t H, float *out, const float *S_q,
-                                 int8_t *out_q, cudaStream_t s);
+                                 int8_t *out_q, uint32_t *amax, cudaStream_t s);
 cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
-                             int8_t *ctx_q, cudaStream_t s);
+                             int8_t *ctx_q, uint32_t *amax, cudaStream_t s);
 
 // Tensor-core attention (q8_attention_sm100.cu): 3 x TF32 split products with fp32 accumulation in TMEM.
 bool attention_tc_supported(const float *qkv, int64_t S, int64_t heads, const float *ctx, const int8_t *ctx_q);
 cudaError_t launch_attention_tc(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
-                                int8_t *ctx_q, cudaStream_t s);
+                                int8_t *ctx_q, uint32_t *amax, cudaStream_t s);
 void set_attention_tensor_cores(bool enable);
 int32_t *attention_status_word();  // device word that receives Q8_ERR_TIMEOUT from the tensor-core attention kernel
 
@@ -95,11 +100,13 @@ void set_gemm_epilogue_warps(int warps);  // 0 automatic, 8 or 16
 cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s);  // q8_gemm_sm100.cu
 cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_generic.cu
 
+
 // The body of q8_linear / q8_linear_generic: validates, quantises X into `workspace`, runs the GEMM (q8_api.cu).
 q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const float *S_x, const float *bias, int act,
                       float *Y, int64_t M, int64_t N, int64_t K, void *workspace, size_t workspace_bytes,
                       int8_t *dbg_Xq, int32_t *dbg_acc, void *stream, bool force_generic, int8_t *Yq = nullptr,
-                      const float *S_y = nullptr, int64_t w_seg = 0);
+                      const float *S_y = nullptr, int64_t w_seg = 0, const uint32_t *x_absmax = nullptr,
+                      uint32_t *y_absmax = nullptr);
 
 // ---- programmatic dependent launch
 // A kernel launched with launch_overlapping_tail() may be scheduled while the kernel before it in the stream is
@@ -164,6 +171,15 @@ __device__ __forceinline__ float finish_output(int32_t acc_plus_bias, float inv_
 {
     float y = __fmul_rn(__int2float_rn(acc_plus_bias), inv_S_out);
     return act == Q8_ACT_GELU ? gelu_erf(y) : y;
+}
+
+// Folds a warp's running max|.| into a device word: non-negative floats order like their bit patterns, NaN never
+// enters (fmaxf drops it), +Inf propagates; nothing is written for an all-zero warp.
+__device__ __forceinline__ void warp_fold_absmax(float m, uint32_t *word)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0 && m > 0.0f) atomicMax(word, __float_as_uint(m));
 }
 
 __device__ __forceinline__ int32_t add_wrap(int32_t a, int32_t b)

@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_kernel(const float *
                                                                    const float *__restrict__ gamma,
                                                                    const float *__restrict__ beta, float eps, int64_t H,
                                                                    float *__restrict__ out, const float *__restrict__ S_q,
-                                                                   int8_t *__restrict__ out_q)
+                                                                   int8_t *__restrict__ out_q, uint32_t *__restrict__ amax)
 {
     extern __shared__ float row[];
     __shared__ float scratch[kLnThreads / 32];
@@ -58,13 +58,16 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_kernel(const float *
     const float var = block_sum(q, scratch) / (float)H;
     const float rstd = 1.0f / sqrtf(var + eps);
     const float Sq = out_q ? __ldg(S_q) : 1.0f;
+    float am = 0.0f;
     for (int64_t h = threadIdx.x; h < H; h += kLnThreads) {
         const float g = gamma ? gamma[h] : 1.0f, b = beta ? beta[h] : 0.0f;
         const float y = (row[h] - mean) * rstd * g + b;
+        am = fmaxf(am, fabsf(y));
         if (out) out[base + h] = y;
         // the same fp32 value, quantised for the next quantised layer (Eq. 1 at that layer's scale)
         if (out_q) out_q[base + h] = (int8_t)quantize_value(y, Sq);
     }
+    if (amax) warp_fold_absmax(am, amax);  // max|y| for a dynamically quantised consumer (Sec. 4.1)
 }
 
 // Vector form for H % 4 == 0, H <= 4096 and 16-byte aligned rows: the row lives in registers (up to four
@@ -76,7 +79,7 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_vec_kernel(const flo
                                                                        const float *__restrict__ beta, float eps,
                                                                        int64_t H, float *__restrict__ out,
                                                                        const float *__restrict__ S_q,
-                                                                       int8_t *__restrict__ out_q)
+                                                                       int8_t *__restrict__ out_q, uint32_t *__restrict__ amax)
 {
     __shared__ float scratch[kLnThreads / 32];
     const int64_t base4 = (int64_t)blockIdx.x * (H >> 2);
@@ -108,6 +111,7 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_vec_kernel(const flo
     const float var = block_sum(q, scratch) / (float)H;
     const float rstd = 1.0f / sqrtf(var + eps);
     const float Sq = out_q ? __ldg(S_q) : 1.0f;
+    float am = 0.0f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int c = threadIdx.x + kLnThreads * i;
@@ -119,9 +123,11 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_vec_kernel(const flo
         y.y = (v[i].y - mean) * rstd * g.y + b.y;
         y.z = (v[i].z - mean) * rstd * g.z + b.z;
         y.w = (v[i].w - mean) * rstd * g.w + b.w;
+        am = fmaxf(fmaxf(am, fmaxf(fabsf(y.x), fabsf(y.y))), fmaxf(fabsf(y.z), fabsf(y.w)));
         if (out) reinterpret_cast<float4 *>(out)[base4 + c] = y;
         if (out_q) reinterpret_cast<uint32_t *>(out_q)[base4 + c] = quantize_pack4(y.x, y.y, y.z, y.w, Sq);
     }
+    if (amax) warp_fold_absmax(am, amax);
 }
 
 // One warp per row for H <= 1024 (BERT's hidden sizes): up to eight float4 per lane, both moments reduced with
@@ -133,12 +139,13 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_warp_kernel(const fl
                                                                         const float *__restrict__ beta, float eps,
                                                                         int64_t rows, int64_t H, float *__restrict__ out,
                                                                         const float *__restrict__ S_q,
-                                                                        int8_t *__restrict__ out_q)
+                                                                        int8_t *__restrict__ out_q, uint32_t *__restrict__ amax)
 {
     grid_dependency_wait();  // launched so that its start may overlap the tail of the kernel before it
     const int lane = threadIdx.x & 31;
     const int n4 = (int)(H >> 2);
     const float Sq = out_q ? __ldg(S_q) : 1.0f;
+    float am = 0.0f;  // running max|y| of this lane over all rows of the warp
     // the grid is sized to the device and every warp walks rows with a grid stride (no partial last wave)
     for (int64_t row = (int64_t)blockIdx.x * (kLnThreads / 32) + (threadIdx.x >> 5); row < rows;
          row += (int64_t)gridDim.x * (kLnThreads / 32)) {
@@ -183,10 +190,12 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_warp_kernel(const fl
         y.y = (v[i].y - mean) * rstd * g.y + b.y;
         y.z = (v[i].z - mean) * rstd * g.z + b.z;
         y.w = (v[i].w - mean) * rstd * g.w + b.w;
+        am = fmaxf(fmaxf(am, fmaxf(fabsf(y.x), fabsf(y.y))), fmaxf(fabsf(y.z), fabsf(y.w)));
         if (out) reinterpret_cast<float4 *>(out)[base4 + c] = y;
         if (out_q) reinterpret_cast<uint32_t *>(out_q)[base4 + c] = quantize_pack4(y.x, y.y, y.z, y.w, Sq);
     }
     }
+    if (amax) warp_fold_absmax(am, amax);  // one atomic per warp: max|y| for a dynamically quantised consumer (Sec. 4.1)
 }
 
 // ------------------------------------------------------------------ self-attention, head dimension 64, no mask
@@ -203,7 +212,8 @@ __device__ __forceinline__ int own_index(int t, int a) { return 2 * t + (a & 1) 
 
 __global__ void __launch_bounds__(256) attention_kernel(const float *__restrict__ qkv, int64_t S, int64_t H,
                                                         float scale, float *__restrict__ ctx,
-                                                        const float *__restrict__ S_q, int8_t *__restrict__ ctx_q)
+                                                        const float *__restrict__ S_q, int8_t *__restrict__ ctx_q,
+                                                        uint32_t *__restrict__ amax)
 {
     extern __shared__ __align__(16) float attn_smem[];
     float(*Qt)[kPitch] = reinterpret_cast<float(*)[kPitch]>(attn_smem);                    // Qt[d][i]
@@ -322,12 +332,14 @@ __global__ void __launch_bounds__(256) attention_kernel(const float *__restrict_
 
     const int64_t obase = seq * S * H + head * kD;
     const float Sq = ctx_q ? __ldg(S_q) : 1.0f;
+    float am = 0.0f;
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
         const int64_t i = q0 + own_index(ty, a);
         if (i >= S) continue;
         const float inv = 1.0f / l[a];
         const float y0 = o[a][0] * inv, y1 = o[a][1] * inv, y2 = o[a][2] * inv, y3 = o[a][3] * inv;
+        am = fmaxf(fmaxf(am, fmaxf(fabsf(y0), fabsf(y1))), fmaxf(fabsf(y2), fabsf(y3)));
         const int64_t at = obase + i * H + 2 * tx;
         if (ctx) {
             *reinterpret_cast<float2 *>(ctx + at) = make_float2(y0, y1);
@@ -340,13 +352,14 @@ __global__ void __launch_bounds__(256) attention_kernel(const float *__restrict_
             ctx_q[at + 33] = (int8_t)quantize_value(y3, Sq);
         }
     }
+    if (amax) warp_fold_absmax(am, amax);
 }
 
 }  // namespace
 
 cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r2, const float *gamma,
                                  const float *beta, float eps, int64_t rows, int64_t H, float *out, const float *S_q,
-                                 int8_t *out_q, cudaStream_t s)
+                                 int8_t *out_q, uint32_t *amax, cudaStream_t s)
 {
     if (rows <= 0 || H <= 0) return cudaSuccess;
     auto al16 = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
@@ -359,21 +372,22 @@ cudaError_t launch_add_layernorm(const float *x, const float *r1, const float *r
         const int64_t cap = (int64_t)(sms > 0 ? sms : 148) * kLnCtasPerSm;
         const unsigned blocks = (unsigned)(want < cap ? want : cap);
         return launch_overlapping_tail(add_layernorm_warp_kernel, dim3(blocks), dim3(kLnThreads), 0, s, x, r1, r2, gamma, beta,
-                                       eps, rows, H, out, S_q, out_q);
+                                       eps, rows, H, out, S_q, out_q, amax);
     } else if (vec) {
-        add_layernorm_vec_kernel<<<(unsigned)rows, kLnThreads, 0, s>>>(x, r1, r2, gamma, beta, eps, H, out, S_q, out_q);
+        add_layernorm_vec_kernel<<<(unsigned)rows, kLnThreads, 0, s>>>(x, r1, r2, gamma, beta, eps, H, out, S_q, out_q, amax);
     } else {
         add_layernorm_kernel<<<(unsigned)rows, kLnThreads, (size_t)H * sizeof(float), s>>>(x, r1, r2, gamma, beta, eps,
-                                                                                           H, out, S_q, out_q);
+                                                                                           H, out, S_q, out_q, amax);
     }
     return cudaGetLastError();
 }
 
 cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t heads, float *ctx, const float *S_q,
-                             int8_t *ctx_q, cudaStream_t s)
+                             int8_t *ctx_q, uint32_t *amax, cudaStream_t s)
 {
     if (B <= 0 || S <= 0 || heads <= 0) return cudaSuccess;
-    if (attention_tc_supported(qkv, S, heads, ctx, ctx_q)) return launch_attention_tc(qkv, B, S, heads, ctx, S_q, ctx_q, s);
+    if (attention_tc_supported(qkv, S, heads, ctx, ctx_q))
+        return launch_attention_tc(qkv, B, S, heads, ctx, S_q, ctx_q, amax, s);
     static bool attr_set[64] = {};  // opt-in shared-memory size: per device, per function
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -385,7 +399,7 @@ cudaError_t launch_attention(const float *qkv, int64_t B, int64_t S, int64_t hea
         attr_set[dev] = true;
     }
     dim3 grid((unsigned)((S + kTile - 1) / kTile), (unsigned)heads, (unsigned)B);
-    attention_kernel<<<grid, 256, kAttnSmemBytes, s>>>(qkv, S, heads * kD, 1.4426950408889634f / 8.0f, ctx, S_q, ctx_q);
+    attention_kernel<<<grid, 256, kAttnSmemBytes, s>>>(qkv, S, heads * kD, 1.4426950408889634f / 8.0f, ctx, S_q, ctx_q, amax);
     return cudaGetLastError();
 }
 

@@ -159,6 +159,40 @@ class Q8BertEncoder:
                 q8.q8_add_layernorm(bf["f2"], bf["h1"], eps=LN_EPS, out=bf["h"])
         return bf["h"]
 
+    def forward_dynamic_fused(self, ids: torch.Tensor, B: int, S: int) -> torch.Tensor:
+        """Dynamic quantisation (Sec. 4.1: every FC derives its scale from max|x| of the incoming tensor) without a
+        single stand-alone abs-max pass: every kernel that produces an FC input (LayerNorm, attention, FFN1's
+        epilogue) also folds max|output| into a device word, and the consuming FC takes 127 / that maximum.  Same
+        Int8 tensors and the same result, bit for bit, as forward(scales="dynamic")."""
+        T = B * S
+        bf = self._buffers(T)
+        if "amax" not in bf:
+            bf["amax"] = torch.zeros(4 * self.L, dtype=torch.int32, device=self.device)
+        amax = bf["amax"]
+        amax.zero_()                      # the words only ever rise: start every forward at zero (one memset)
+        word = lambda l, i: amax[4 * l + i: 4 * l + i + 1]
+        pos_ids = torch.arange(S, dtype=torch.int32, device=self.device).repeat(B)
+        typ_ids = torch.zeros(T, dtype=torch.int32, device=self.device)
+        q8.q8_embedding(ids, self.word, self.S_word, out=bf["ew"], dev_status=bf["status"])
+        q8.q8_embedding(pos_ids, self.pos, self.S_pos, out=bf["ep"], dev_status=bf["status"])
+        q8.q8_embedding(typ_ids, self.typ, self.S_typ, out=bf["et"], dev_status=bf["status"])
+        q8.q8_add_layernorm_absmax(bf["ew"], word(0, 0), bf["ep"], bf["et"], eps=LN_EPS, out=bf["h"])
+        for l in range(self.L):
+            p = self.layers[l]
+            lin = lambda name, X, xw, Y, yw=None: q8.q8_linear_dyn(X, xw, p[name]["Wq"], p[name]["S_w"], p[name]["b"],
+                                                                   p[name]["act"], Y=Y, y_absmax=yw, workspace=bf["ws"])
+            lin("qkv", bf["h"], word(l, 0), bf["qkv"])
+            q8.q8_attention_absmax(bf["qkv"], B, S, self.heads, word(l, 1), ctx=bf["ctx"])
+            lin("attn_out", bf["ctx"], word(l, 1), bf["ao"])
+            q8.q8_add_layernorm_absmax(bf["ao"], word(l, 2), bf["h"], eps=LN_EPS, out=bf["h1"])
+            lin("ffn1", bf["h1"], word(l, 2), bf["f"], word(l, 3))
+            lin("ffn2", bf["f"], word(l, 3), bf["f2"])
+            if l + 1 < self.L:
+                q8.q8_add_layernorm_absmax(bf["f2"], word(l + 1, 0), bf["h1"], eps=LN_EPS, out=bf["h"])
+            else:
+                q8.q8_add_layernorm(bf["f2"], bf["h1"], eps=LN_EPS, out=bf["h"])
+        return bf["h"]
+
     def capture(self, ids: torch.Tensor, B: int, S: int, fused: bool = True):
         """Captures one static-scale forward into a CUDA graph (the forward is a fixed sequence of launches on
         fixed buffers, and for small batches the host cannot issue them as fast as the GPU runs them).
@@ -172,6 +206,8 @@ class Q8BertEncoder:
         return graph, out
 
     def launches_per_forward(self, scales: str = "static", fused: bool = False) -> int:
+        if fused and scales == "dynamic":
+            return 4 + self.L * 11          # per layer: 4 x (quantise + GEMM), attention, two LayerNorms
         if fused:
             return 4 + self.L * 7
         per_fc = 2 if scales == "static" else (3 if scales == "dynamic" else 5)

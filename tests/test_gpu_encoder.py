@@ -245,3 +245,90 @@ def test_fused_forward_is_bit_identical_to_the_unfused_one():
         torch.cuda.synchronize()
         replayed = out.clone()
         assert torch.equal(replayed, enc.forward(ids, B, S, scales="static"))
+
+
+# ------------------------------------------------------------------ dynamic quantisation with fused abs-max (Sec. 4.1)
+def _word():
+    return torch.zeros(1, dtype=torch.int32, device="cuda")
+
+
+def _bits_of_absmax(t: torch.Tensor) -> int:
+    """IEEE bits of the oracle's max|.| over the tensor the GPU actually stored."""
+    return int(np.float32(o.absmax(t.cpu().numpy())).view(np.uint32))
+
+
+@pytest.mark.parametrize("rows,H", [(37, 96), (300, 768), (5, 1000), (3, 2048), (3, 1001), (2000, 1024)])
+def test_layernorm_folds_the_absmax_of_what_it_stores(rows, H):
+    x = synth.activation(rows, H, 3400 + H)
+    r1 = synth.activation(rows, H, 3401 + H)
+    w = _word()
+    out = q8.q8_add_layernorm_absmax(dev(x), w, dev(r1))
+    assert torch.equal(out, q8.q8_add_layernorm(dev(x), dev(r1)))           # same values as the plain call
+    assert (w.item() & 0xFFFFFFFF) == _bits_of_absmax(out)
+    # the word only ever rises: a second producer with smaller values leaves it, one with larger values raises it
+    before = w.item()
+    q8.q8_add_layernorm_absmax(dev(x), w, dev(r1), gamma=dev(np.full(H, 0.5, np.float32)))
+    assert w.item() == before
+    big = q8.q8_add_layernorm_absmax(dev(x), w, dev(r1), gamma=dev(np.full(H, 3.0, np.float32)))
+    assert (w.item() & 0xFFFFFFFF) == _bits_of_absmax(big)
+
+
+@pytest.mark.parametrize("B,S,heads,tensor_cores", [(2, 100, 2, True), (1, 384, 4, True), (2, 70, 2, False), (1, 500, 1, True)])
+def test_attention_folds_the_absmax_of_what_it_stores(B, S, heads, tensor_cores):
+    qkv = dev(synth.normal((B * S, 3 * heads * 64), 1.0, 3450 + S))
+    try:
+        q8.q8_tune_attention(tensor_cores)
+        w = _word()
+        ctx = q8.q8_attention_absmax(qkv, B, S, heads, w)
+        assert torch.equal(ctx, q8.q8_attention(qkv, B, S, heads))
+        assert (w.item() & 0xFFFFFFFF) == _bits_of_absmax(ctx)
+    finally:
+        q8.q8_tune_attention(True)
+
+
+@pytest.mark.parametrize("M,N,K,act", [(300, 200, 400, 1), (515, 1030, 144, 0), (4096, 768, 768, 1), (100, 52, 50, 1),
+                                       (20000, 1000, 128, 1)])
+def test_linear_dyn_takes_its_scale_from_a_word_and_reports_its_own_output_absmax(M, N, K, act):
+    """q8_linear_dyn with max|X| supplied by the producer equals q8_linear with its own abs-max pass, bit for bit
+    (and therefore the oracle, which check_linear compares q8_linear with), in two kernels instead of four
+    operations; its y_absmax word is the oracle's max|.| of the stored output."""
+    X = synth.activation(M, K, 3500 + M)
+    Wq, S_w = q8.q8_quantize_weight(dev(synth.weight(N, K, 3501 + M)))
+    b = dev(synth.bias(N, 3502 + M))
+    Xd = dev(X)
+    xw = _word()
+    # the producer here is a LayerNorm that reproduces X: fold max|X| with the library's own abs-max kernel instead
+    _, S_dyn = q8.q8_quantize_activation(Xd)                       # S = 127 / max|X|
+    xw.copy_(torch.from_numpy(np.array([np.float32(o.absmax(X))]).view(np.int32)))
+    ws0, ws1 = q8.new_workspace(M, N, K), q8.new_workspace(M, N, K)
+    xq0, xq1 = (torch.empty((M, K), dtype=torch.int8, device="cuda") for _ in range(2))
+    a0, a1 = (torch.empty((M, N), dtype=torch.int32, device="cuda") for _ in range(2))
+    Y0 = q8.q8_linear(Xd, Wq, S_w, None, b, act, workspace=ws0, dbg_Xq=xq0, dbg_acc=a0)
+    launches_plain = q8.q8_last_launch_info()["launches"]
+    yw = _word()
+    Y1 = q8.q8_linear_dyn(Xd, xw, Wq, S_w, b, act, y_absmax=yw, workspace=ws1, dbg_Xq=xq1, dbg_acc=a1)
+    assert q8.q8_last_launch_info()["launches"] == 2 and launches_plain == 3
+    assert q8.q8_poll_status(ws1) == (q8.Q8_OK, 0)
+    assert torch.equal(xq0, xq1) and torch.equal(a0, a1) and torch.equal(Y0, Y1)
+    assert ws1[4:8].view(torch.float32).item() == S_dyn.item() == ws0[4:8].view(torch.float32).item()
+    assert (yw.item() & 0xFFFFFFFF) == _bits_of_absmax(Y1)
+    ref = o.linear(X, Wq.cpu().numpy(), S_w.item(), None, b.cpu().numpy(), act)
+    assert np.array_equal(xq1.cpu().numpy(), ref["xq"]) and np.array_equal(a1.cpu().numpy(), ref["acc"])
+    assert_close_fp(Y1.cpu().numpy(), ref["y"], "Y")
+    # a word that is still zero (producer never ran) is reported, not divided by
+    q8.q8_linear_dyn(Xd, _word(), Wq, S_w, b, act, workspace=ws1)
+    assert q8.q8_poll_status(ws1)[0] == q8.Q8_ERR_SCALE
+
+
+def test_dynamic_forward_without_absmax_passes_equals_the_unfused_dynamic_forward():
+    """Sec. 4.1 end to end: the forward whose producers fold max|y| (no stand-alone abs-max pass, no memset per FC)
+    gives the same bits as the forward in which every q8_linear computes its own dynamic scale."""
+    dims = dict(synth.BERT_BASE, layers=3)
+    enc = enc_mod.Q8BertEncoder(dims, config=3)
+    B, S = 4, 128
+    ids = enc_mod.random_ids(B * S, dims["vocab"], 3)
+    want = enc.forward(ids, B, S, scales="dynamic").clone()
+    got = enc.forward_dynamic_fused(ids, B, S)
+    assert torch.equal(got, want)
+    assert enc.poll() == ((q8.Q8_OK, 0), (q8.Q8_OK, 0))
+    assert enc.launches_per_forward("dynamic", fused=True) < enc.launches_per_forward("dynamic")
