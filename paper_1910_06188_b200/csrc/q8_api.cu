@@ -101,6 +101,10 @@ q8_status linear_impl(const float *X, const int8_t *Wq, const float *S_w, const 
         // derives the scale from it, publishes it in the header and quantises; it also starts the status word at zero.
         Q8_CUDA_TRY(launch_quantize_dynamic(X, M * K, x_absmax, &hdr->S_x_dyn, &hdr->status, Xq, dbg_Xq, s, true));
         last_launch_info().launches += 1;
+    } else if (quantize_dynamic_small_supported(X, M * K, Xq, dbg_Xq)) {
+        // a small activation (up to 256 x 768): abs-max, scale and Eq. 1 in one launch of one cluster, no memset
+        Q8_CUDA_TRY(launch_quantize_dynamic_small(X, M * K, &hdr->S_x_dyn, &hdr->status, Xq, dbg_Xq, s));
+        last_launch_info().launches += 1;
     } else {
         Q8_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), s));
         Q8_CUDA_TRY(launch_absmax(X, M * K, &hdr->absmax_bits, s));

@@ -173,6 +173,86 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
     }
 }
 
+// Dynamic scale and Eq. 1 in ONE launch for a small activation (Sec. 4.1; e.g. one 128-token batch): a single
+// cluster of 8 CTAs holds the whole tensor in registers (up to 12 float4 per thread), so the tensor is read once.
+// Each CTA reduces max|x| of its share, the 8 partial maxima are exchanged through distributed shared memory
+// (one cluster barrier), every thread derives the same S = 127 / max|x| and quantises the values it holds.
+// CTA 0 publishes S and sets the call's status word (0, or the Q8_ERR_SCALE bit for a zero / infinite maximum).
+constexpr int kDqCluster = 8, kDqThreads = 512, kDqVecPerThread = 12;
+constexpr int64_t kDqMaxElems = (int64_t)kDqCluster * kDqThreads * kDqVecPerThread * 4;  // 196608 = 256 x 768
+
+__global__ void __launch_bounds__(kDqThreads) quantize_dynamic_cluster_kernel(const float *__restrict__ x, int64_t n,
+                                                                              float *__restrict__ S_out,
+                                                                              int32_t *__restrict__ status,
+                                                                              int8_t *__restrict__ xq,
+                                                                              int8_t *__restrict__ xq_copy)
+{
+    grid_dependency_wait();
+    __shared__ float warp_max[kDqThreads / 32];
+    __shared__ float cta_max, all_max;
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int64_t n4 = n >> 2;  // n % 4 == 0 (checked by the host)
+    const float4 *x4 = reinterpret_cast<const float4 *>(x);
+    const int64_t first = (int64_t)rank * kDqThreads + threadIdx.x;
+    constexpr int64_t kStride = (int64_t)kDqCluster * kDqThreads;
+    float4 v[kDqVecPerThread];
+    float m = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kDqVecPerThread; ++i) {
+        const int64_t idx = first + i * kStride;
+        v[i] = idx < n4 ? __ldg(x4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        m = absmax4(m, v[i]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        m = threadIdx.x < kDqThreads / 32 ? warp_max[threadIdx.x] : 0.0f;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (threadIdx.x == 0) cta_max = m;
+    }
+    // every CTA's partial maximum is in place before any CTA reads its peers'
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (threadIdx.x < 32) {
+        float p = 0.0f;
+        if (threadIdx.x < kDqCluster) {
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;"
+                         : "=r"(remote)
+                         : "r"((uint32_t)__cvta_generic_to_shared(&cta_max)), "r"((uint32_t)threadIdx.x));
+            asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(p) : "r"(remote) : "memory");
+        }
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) p = fmaxf(p, __shfl_xor_sync(0xffffffffu, p, o));
+        if (threadIdx.x == 0) all_max = p;
+    }
+    // no CTA may exit (and give up its shared memory) while a peer can still read it
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    __syncthreads();
+    const float a = all_max;
+    const bool bad = !(a > 0.0f) || isinf(a);
+    const float S = bad ? 1.0f : __fdiv_rn(127.0f, a);
+    if (rank == 0 && threadIdx.x == 0) {
+        *S_out = S;
+        if (status) *status = bad ? (1 << Q8_ERR_SCALE) : 0;  // first kernel of the call: starts the status word
+    }
+    uint32_t *q4 = reinterpret_cast<uint32_t *>(xq);
+    uint32_t *c4 = reinterpret_cast<uint32_t *>(xq_copy);
+#pragma unroll
+    for (int i = 0; i < kDqVecPerThread; ++i) {
+        const int64_t idx = first + i * kStride;
+        if (idx < n4) {
+            const uint32_t q = quantize_pack4(v[i], S);
+            q4[idx] = q;
+            if (xq_copy) c4[idx] = q;
+        }
+    }
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // ------------------------------------------------------------------ Eq. 4
 __global__ void ema_update_kernel(CalibState *st, float decay)
 {
@@ -337,6 +417,31 @@ cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *a
                                                                                  S_out, status, clear_word);
     }
     return cudaGetLastError();
+}
+
+bool quantize_dynamic_small_supported(const float *x, int64_t n, const int8_t *xq, const int8_t *xq_copy)
+{
+    return n > 0 && n <= kDqMaxElems && (n & 3) == 0 && aligned16(x) && aligned16(xq) &&
+           (xq_copy == nullptr || aligned16(xq_copy));
+}
+
+cudaError_t launch_quantize_dynamic_small(const float *x, int64_t n, float *S_out, int32_t *status, int8_t *xq,
+                                          int8_t *xq_copy, cudaStream_t s)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kDqCluster);
+    cfg.blockDim = dim3(kDqThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kDqCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, quantize_dynamic_cluster_kernel, x, n, S_out, status, xq, xq_copy);
 }
 
 cudaError_t launch_fake_quantize(const float *x, int64_t n, const float *S, float *xhat, cudaStream_t s)

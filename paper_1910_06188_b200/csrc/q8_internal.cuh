@@ -71,6 +71,11 @@ cudaError_t launch_quantize(const float *x, int64_t n, const float *S, int8_t *x
 cudaError_t launch_quantize_dynamic(const float *x, int64_t n, const uint32_t *absmax_bits, float *S_out,
                                     int32_t *status, int8_t *xq, int8_t *xq_copy, cudaStream_t s,
                                     bool clear_status = false);
+// Small tensors (n <= 196608, n % 4 == 0, 16-byte aligned): abs-max, scale and Eq. 1 in one launch of one cluster.
+// *status (may be NULL) is SET (0 or the Q8_ERR_SCALE bit), not OR-ed into.
+bool quantize_dynamic_small_supported(const float *x, int64_t n, const int8_t *xq, const int8_t *xq_copy);
+cudaError_t launch_quantize_dynamic_small(const float *x, int64_t n, float *S_out, int32_t *status, int8_t *xq,
+                                          int8_t *xq_copy, cudaStream_t s);
 cudaError_t launch_ema_update(CalibState *st, float decay, cudaStream_t s);
 cudaError_t launch_fake_quantize(const float *x, int64_t n, const float *S, float *xhat, cudaStream_t s);
 cudaError_t launch_embedding(const int32_t *ids, int64_t T, const int8_t *Eq, const float *S_e, int64_t V,

@@ -307,7 +307,8 @@ def test_linear_dyn_takes_its_scale_from_a_word_and_reports_its_own_output_absma
     launches_plain = q8.q8_last_launch_info()["launches"]
     yw = _word()
     Y1 = q8.q8_linear_dyn(Xd, xw, Wq, S_w, b, act, y_absmax=yw, workspace=ws1, dbg_Xq=xq1, dbg_acc=a1)
-    assert q8.q8_last_launch_info()["launches"] == 2 and launches_plain == 3
+    # q8_linear itself needs a memset-free single quantise launch only for small activations (one cluster holds them)
+    assert q8.q8_last_launch_info()["launches"] == 2 and launches_plain == (2 if M * K <= 196608 and M * K % 4 == 0 else 3)
     assert q8.q8_poll_status(ws1) == (q8.Q8_OK, 0)
     assert torch.equal(xq0, xq1) and torch.equal(a0, a1) and torch.equal(Y0, Y1)
     assert ws1[4:8].view(torch.float32).item() == S_dyn.item() == ws0[4:8].view(torch.float32).item()

@@ -209,6 +209,32 @@ def test_device_side_errors_are_returned_as_codes():
     assert e.value.status == q8.Q8_ERR_ARG
 
 
+@pytest.mark.parametrize("M,K,N", [(128, 768, 768), (256, 768, 96), (1, 16, 8), (37, 96, 40), (4, 48, 32), (255, 768, 64)])
+def test_small_dynamic_layer_is_two_launches_and_matches_the_oracle(M, K, N):
+    """A small activation (up to 256 x 768 values) is abs-maxed, scaled and quantised by one cluster in one launch
+    (Sec. 4.1 + Eq. 1), so the whole dynamic layer is two kernels; same bits as the oracle, call after call."""
+    X = synth.activation(M, K, seed=700 + M)
+    W = synth.weight(N, K, seed=701 + M)
+    b = synth.bias(N, seed=702 + M)
+    for _ in range(2):
+        info = check_linear(X, W, b, act=1)
+        assert info["launches"] == 2
+    # all-zero and non-finite activations: scale forced to 1, flagged, no NaN in the Int8 tensor
+    Wq, S_w = q8.q8_quantize_weight(dev(W))
+    ws = q8.new_workspace(M, N, K)
+    xq = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    q8.q8_linear(torch.zeros((M, K), device="cuda"), Wq, S_w, None, dev(b), 0, workspace=ws, dbg_Xq=xq)
+    assert q8.q8_poll_status(ws)[0] == q8.Q8_ERR_SCALE and not xq.any()
+    Xi = dev(X).clone()
+    Xi[0, 0] = float("inf")
+    Xi[0, 1] = float("nan")
+    q8.q8_linear(Xi, Wq, S_w, None, dev(b), 0, workspace=ws, dbg_Xq=xq)
+    assert q8.q8_poll_status(ws)[0] == q8.Q8_ERR_SCALE
+    assert np.array_equal(xq.cpu().numpy(), o.quantize(Xi.cpu().numpy(), 1.0))
+    q8.q8_linear(dev(X), Wq, S_w, None, dev(b), 0, workspace=ws)        # and the next call starts clean
+    assert q8.q8_poll_status(ws) == (q8.Q8_OK, 0)
+
+
 # ------------------------------------------------------------------ the paper-shaped configurations
 def test_config_single_layer_dynamic():
     """X [128 x 768] with x8 outliers, W [768 x 768], bias; dynamic S_x (Sec. 4.1)."""
