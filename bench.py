@@ -40,10 +40,13 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of the tcgen05 GEMM per launch on the BERT-Large FC set, from the
 # ncu captures summarised in profiles/gemm_tcgen05_dram_traffic_m24576.md (one layer resident per capture).  Below the
 # algorithmic bytes because part of each output is still dirty in the 126 MB L2 when the kernel ends.
-GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 269126912, "attn_out": 66280448, "ffn1": 371268608, "ffn2": 163438592}}
+GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 270513664, "attn_out": 67436288, "ffn1": 372471296, "ffn2": 164332800}}
 NOMINAL_INT8_OVER_BF16 = 2.0  # dense tensor peak ratio int8 : bf16 (4.5 : 2.25 POPS nominal)
-GEMM_REPS = 4  # launches per event pair in the per-kernel pass
-EMB_REPS = 4   # embedding gathers per event pair in the per-kernel pass
+GEMM_REPS = 4   # launches per event pair in the per-kernel pass
+QUANT_REPS = 4  # times each group of equal-sized quantise passes is repeated per event pair
+EMB_REPS = 4    # embedding gathers per event pair in the per-kernel pass
+EMB_TABLES = 6  # copies of the embedding table the L2-cold gather figure rotates over (6 x 31 MB > L2)
+REPLAY_SAMPLES = 100  # individually timed replays of the step for the median / best figures
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -143,7 +146,8 @@ def run_reference(args):
     from oracle import q8_oracle as o  # the one place besides cpu_baseline where bench.py runs the oracle
 
     cfg_index, dims, desc = WORKLOADS[args.workload]
-    rows = args.reference_rows
+    M_full = dims["batch"] * dims["seq"]
+    rows = M_full if args.reference_rows <= 0 else min(args.reference_rows, M_full)
     layers = []
     for i, (name, K, N, act) in enumerate(synth.fc_set(dims["hidden"], dims["ffn"])):
         X = synth.activation(rows, K, synth.seed_for(cfg_index, 10 * i))
@@ -158,20 +162,28 @@ def run_reference(args):
         for L in layers:
             o.linear(L["X"], L["Wq"], L["S_w"], L["S_x"], L["b"], L["act"])
 
-    for _ in range(args.warmup):
-        step()
+    # One step is the whole workload (all token rows of the four layers), which takes the oracle seconds; the
+    # requested warm-up and step counts are cut so that the run stays within --reference-budget-s seconds.
     t0 = time.perf_counter()
-    for _ in range(args.steps):
+    step()
+    first = time.perf_counter() - t0
+    budget = max(args.reference_budget_s - first, first)
+    steps = max(1, min(args.steps, int(budget / first)))
+    warm_done = 1
+    t0 = time.perf_counter()
+    for _ in range(steps):
         step()
-    dt = (time.perf_counter() - t0) / args.steps
+    dt = (time.perf_counter() - t0) / steps
     value = ops / dt / 1e12
     cores = os.cpu_count()
-    sample = f"{rows} of {dims['batch'] * dims['seq']} token rows of each of the 4 FC layers per step"
+    sample = f"{rows} of {M_full} token rows of each of the 4 FC layers per step, {steps} timed step(s) after {warm_done} warm-up"
     line = {
         "impl": "reference", "metric": "q8_linear_int8_tops", "value": value, "unit": "TOPS", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "steps": steps, "warmup": warm_done, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": args.workload, "description": desc, "sample": sample},
+        "config": {"workload": args.workload, "description": desc, "sample": sample,
+                   "steps_requested": args.steps, "warmup_requested": args.warmup,
+                   "tokens_per_step": rows},
         "cpu_baseline": {"value": value, "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -196,6 +208,9 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     q8.load()
+
+    if args.profile_mode and args.encoder_kernel:
+        return profile_encoder_kernel(args, torch, q8)
 
     cfg_index, dims, desc = WORKLOADS[args.workload]
     # weak scaling: every rank owns one full batch of M tokens (rows are independent given static
@@ -310,6 +325,20 @@ def run_ours(args):
         ev1.record(stream)
         barrier()
         ms = ev0.elapsed_time(ev1)
+        # the same step, each repetition between its own pair of events (no host synchronisation in between):
+        # median and best of REPLAY_SAMPLES beside the mean of the K-step region
+        per_step_ms = []
+        if not args.profile_mode:
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(REPLAY_SAMPLES + 1)]
+            marks[0].record(stream)
+            for i in range(REPLAY_SAMPLES):
+                if step_graph is not None:
+                    step_graph.replay()
+                else:
+                    step()
+                marks[i + 1].record(stream)
+            barrier()
+            per_step_ms = [marks[i].elapsed_time(marks[i + 1]) for i in range(REPLAY_SAMPLES)]
         if step_graph is not None:
             # the same K steps launched eagerly from the host, reported beside the graph-replayed figure
             ev0.record(stream)
@@ -323,6 +352,13 @@ def run_ours(args):
         nl = len(layers)
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(nl)]
         t_quant, t_gemm = [0.0] * nl, [0.0] * nl
+        # FFN1 handing its GELU output to FFN2 as Int8 only (Eq. 1 at FFN2's Eq. 4 scale, fused into the epilogue)
+        i8 = next((i for i, L in enumerate(layers) if L["name"] == "ffn1"), None)
+        i8_consumer = next((L for L in layers if L["name"] == "ffn2"), None)
+        t_i8 = 0.0
+        ev_i0, ev_i1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev_c0, ev_c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_emb_cold = 0.0
         ev_e0, ev_e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_emb = 0.0
         ksteps = 0 if args.profile_mode else min(args.steps, 50)
@@ -335,8 +371,24 @@ def run_ours(args):
         # The launches between two events are replayed from a CUDA graph, so the events see device time without
         # host gaps: each layer's GEMM_REPS back-to-back GEMM launches, each group of quantise passes, and
         # EMB_REPS embedding gathers that alternate between two output buffers (together larger than L2).
-        gemm_graphs, quant_graphs, emb_graph = [], {}, None
+        gemm_graphs, quant_graphs, emb_graph, i8_graph, emb_cold_graph = [], {}, None, None, None
         emb_out2 = torch.empty_like(emb_out) if ksteps > 0 else None
+        Yq_i8 = None
+        if ksteps > 0 and i8 is not None and i8_consumer is not None:
+            Yq_i8 = torch.empty((layers[i8]["M"], layers[i8]["N"]), dtype=torch.int8, device=dev)
+        else:
+            i8 = None
+        # L2-cold gather: the tokens of the batch look their rows up in EMB_TABLES copies of the table in turn
+        Eq_copies = [Eq] + [Eq.clone() for _ in range(EMB_TABLES - 1)] if ksteps > 0 else []
+
+        def run_i8():
+            L = layers[i8]
+            for _ in range(GEMM_REPS):
+                q8.q8_linear_q_requant(L["Xq"], L["S_x"], L["Wq"], L["S_w"], L["bd"], L["act"], i8_consumer["S_x"], Yq=Yq_i8)
+
+        def run_emb_cold():
+            for r in range(EMB_TABLES):
+                q8.q8_embedding(ids, Eq_copies[r], S_e, out=emb_out if r % 2 == 0 else emb_out2)
         if not args.no_graph and ksteps > 0:
             try:
                 for L in layers:
@@ -348,9 +400,19 @@ def run_ours(args):
                 for k, members in groups.items():
                     g = torch.cuda.CUDAGraph()
                     with torch.cuda.graph(g, capture_error_mode="thread_local"):
-                        for i in members:
-                            q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
+                        for _ in range(QUANT_REPS):
+                            for i in members:
+                                q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
                     quant_graphs[k] = g
+                if i8 is not None:
+                    run_i8()
+                    i8_graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(i8_graph, capture_error_mode="thread_local"):
+                        run_i8()
+                run_emb_cold()
+                emb_cold_graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(emb_cold_graph, capture_error_mode="thread_local"):
+                    run_emb_cold()
                 emb_graph = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(emb_graph, capture_error_mode="thread_local"):
                     for r in range(EMB_REPS):
@@ -358,7 +420,7 @@ def run_ours(args):
                 torch.cuda.synchronize()
             except Exception as ex:
                 print(f"[bench] CUDA graph capture of the per-kernel pass failed ({ex}); timing eager launches", file=sys.stderr)
-                gemm_graphs, quant_graphs, emb_graph = [], {}, None
+                gemm_graphs, quant_graphs, emb_graph, i8_graph, emb_cold_graph = [], {}, None, None, None
         for _ in range(ksteps):
             ev_e0.record(stream)
             if emb_graph is not None:
@@ -372,8 +434,9 @@ def run_ours(args):
                 if k in quant_graphs:
                     quant_graphs[k].replay()
                 else:
-                    for i in members:
-                        q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
+                    for _ in range(QUANT_REPS):
+                        for i in members:
+                            q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
                 gev[k][1].record(stream)
             for i, L in enumerate(layers):
                 evs[i][1].record(stream)
@@ -383,11 +446,27 @@ def run_ours(args):
                     for _ in range(GEMM_REPS):  # back to back, so that the event overhead is shared by several launches
                         q8.q8_linear_q(L["Xq"], L["S_x"], L["Wq"], L["S_w"], L["bd"], L["act"], Y=L["Y"])
                 evs[i][2].record(stream)
+            if i8 is not None:
+                ev_i0.record(stream)
+                if i8_graph is not None:
+                    i8_graph.replay()
+                else:
+                    run_i8()
+                ev_i1.record(stream)
+            ev_c0.record(stream)
+            if emb_cold_graph is not None:
+                emb_cold_graph.replay()
+            else:
+                run_emb_cold()
+            ev_c1.record(stream)
             torch.cuda.synchronize()
             t_emb += ev_e0.elapsed_time(ev_e1) / EMB_REPS
+            t_emb_cold += ev_c0.elapsed_time(ev_c1) / EMB_TABLES
+            if i8 is not None:
+                t_i8 += ev_i0.elapsed_time(ev_i1) / GEMM_REPS
             for k, members in groups.items():
                 for i in members:
-                    t_quant[i] += gev[k][0].elapsed_time(gev[k][1]) / len(members)
+                    t_quant[i] += gev[k][0].elapsed_time(gev[k][1]) / (len(members) * QUANT_REPS)
             for i in range(nl):
                 t_gemm[i] += evs[i][1].elapsed_time(evs[i][2]) / GEMM_REPS
         # ---- the same step with its five independent jobs spread over five streams (reported beside `value`)
@@ -551,7 +630,21 @@ def run_ours(args):
                     "layer floor = max(2MNK / Int8 peak, 4MN / store-only rate)",
         }
     emb_ms = t_emb / ksteps
+    emb_cold_ms = t_emb_cold / ksteps
     emb_bytes = 5.0 * M * H + 4.0 * M
+    if i8 is not None:
+        L = layers[i8]
+        im = t_i8 / ksteps
+        go = 2.0 * L["M"] * L["N"] * L["K"]
+        gb = L["M"] * L["K"] + L["N"] * L["K"] + 4 * L["N"] + L["M"] * L["N"]
+        t_tensor = go / (int8_peak * 1e12)
+        by_layer.append({
+            "layer": "ffn1_int8_out", "M": L["M"], "K": L["K"], "N": L["N"], "gemm_us": im * 1e3,
+            "gemm_tops": go / (im * 1e-3) / 1e12, "gemm_frac_int8_peak": go / (im * 1e-3) / 1e12 / int8_peak,
+            "gemm_gbs": gb / (im * 1e-3) / 1e9, "gemm_frac_hbm": gb / (im * 1e-3) / 1e9 / hbm_peak,
+            "gemm_floor_us": t_tensor * 1e6, "gemm_floor_bound": "tensor", "gemm_frac_of_floor": t_tensor / (im * 1e-3),
+            "note": "q8_linear_q_requant: FFN1 with GELU emitting only Int8 at FFN2's scale (1 byte per output); not part of the step",
+        })
     roofline = {
         "kernel": "gemm_tcgen05_kernel (4 launches per step, one per FC layer)",
         "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
@@ -587,7 +680,11 @@ def run_ours(args):
                 "all replayed from CUDA graphs unless --no-graph" % (GEMM_REPS, EMB_REPS),
         "by_layer": by_layer,
         "embedding": {"us": emb_ms * 1e3, "gbs": emb_bytes / (emb_ms * 1e-3) / 1e9,
-                      "frac_hbm": emb_bytes / (emb_ms * 1e-3) / 1e9 / hbm_peak},
+                      "frac_hbm": emb_bytes / (emb_ms * 1e-3) / 1e9 / hbm_peak,
+                      "l2_cold": {"us": emb_cold_ms * 1e3, "gbs": emb_bytes / (emb_cold_ms * 1e-3) / 1e9,
+                                  "frac_hbm": emb_bytes / (emb_cold_ms * 1e-3) / 1e9 / hbm_peak,
+                                  "note": "%d gathers in a row, each from its own copy of the table (together larger than L2), "
+                                          "alternating between two output buffers" % EMB_TABLES}},
     }
 
     # ---- CPU oracle on a bounded sample of the same workload (rank 0, N=1 only)
@@ -613,14 +710,24 @@ def run_ours(args):
         for L in layers:
             L.clear()
         del host_in, host_out, host_emb, emb_out, emb_out2, gemm_graphs, quant_graphs, emb_graph, step_graph
+        del Eq_copies, emb_cold_graph, i8_graph, Yq_i8
         torch.cuda.empty_cache()
         encoder = measure_encoders(args, torch, q8)
         small = measure_small_cases(args, torch, q8)
 
+    srt = sorted(per_step_ms)
     line = {
         "metric": "q8_linear_int8_tops", "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        # per-kernel microseconds first, so that a truncated copy of this line still shows every layer
+        "kernel_us": dict([(b["layer"], round(b["gemm_us"], 2)) for b in by_layer]
+                          + [("quantize_" + b["layer"], round(b["quantize_us"], 2)) for b in by_layer if "quantize_us" in b]
+                          + [("embedding", round(emb_ms * 1e3, 2)), ("embedding_l2_cold", round(emb_cold_ms * 1e3, 2))]),
+        "gemm_frac_nominal_int8_4500": dict((b["layer"], round(b["gemm_tops"] / 4500.0, 4)) for b in by_layer),
+        "step_us": {"mean_of_timed_region": ms_per_step * 1e3,
+                    "median": (statistics.median(srt) * 1e3 if srt else None), "best": (srt[0] * 1e3 if srt else None),
+                    "samples": len(srt), "tops_at_median": (ops * world / (statistics.median(srt) * 1e-3) / 1e12 if srt else None)},
         "config": {
             "workload": args.workload, "description": desc, "tokens_per_step": M * world,
             "tokens_per_s": M * world / (ms_per_step * 1e-3),
@@ -646,6 +753,36 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+    return 0
+
+
+def profile_encoder_kernel(args, torch, q8):
+    """--profile-mode --encoder-kernel K: a few launches of one FP32 support kernel of the encoder (attention or
+    residual + LayerNorm) on seeded synthetic data, for an ncu capture of that kernel alone."""
+    B, S, heads, H = args.profile_batch, args.profile_seq, args.profile_heads, args.profile_heads * 64
+    g = torch.Generator(device="cuda").manual_seed(1)
+    if args.encoder_kernel == "attention":
+        qkv = torch.randn((B * S, 3 * H), device="cuda", generator=g)
+        ctx = torch.empty((B * S, H), device="cuda")
+        fn = lambda: q8.q8_attention(qkv, B, S, heads, ctx=ctx)
+        work, unit = 4.0 * B * heads * S * S * 64, "TFLOP/s"
+    else:
+        x = torch.randn((B * S, H), device="cuda", generator=g)
+        r = torch.randn((B * S, H), device="cuda", generator=g)
+        out = torch.empty_like(x)
+        fn = lambda: q8.q8_add_layernorm(x, r, out=out)
+        work, unit = 12.0 * B * S * H, "TB/s"
+    fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(max(args.steps, 1)):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / max(args.steps, 1)
+    print(json.dumps({"profile_mode": True, "encoder_kernel": args.encoder_kernel, "batch": B, "seq": S, "heads": heads,
+                      "us_per_call": ms * 1e3, "rate": work / (ms * 1e-3) / 1e12, "unit": unit}), flush=True)
     return 0
 
 
@@ -828,7 +965,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-rows", type=int, default=24576,
                     help="token rows per layer for the cpu_baseline sample (default: the whole workload once, ~10 s)")
-    ap.add_argument("--reference-rows", type=int, default=256, help="token rows per layer per step for --impl reference")
+    ap.add_argument("--reference-rows", type=int, default=0,
+                    help="token rows per layer per step for --impl reference (0 = the whole workload, as the GPU arm)")
+    ap.add_argument("--reference-budget-s", type=float, default=150.0,
+                    help="--impl reference cuts its step count so that the run stays within this many seconds")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-encoder", action="store_true", help="skip the whole-encoder tokens/s measurement")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of CUDA graph replays")
@@ -838,6 +978,11 @@ def main():
     ap.add_argument("--layers", default="", help="comma list of FC layers to keep (qkv,attn_out,ffn1,ffn2); default all")
     ap.add_argument("--profile-mode", action="store_true",
                     help="only warm-up + timed steps (no per-kernel pass, e2e or CPU baseline): for ncu captures")
+    ap.add_argument("--encoder-kernel", choices=["attention", "layernorm"], default="",
+                    help="with --profile-mode: launch only this FP32 support kernel of the encoder (--steps times)")
+    ap.add_argument("--profile-batch", type=int, default=8)
+    ap.add_argument("--profile-seq", type=int, default=384)
+    ap.add_argument("--profile-heads", type=int, default=16)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

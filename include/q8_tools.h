@@ -21,8 +21,7 @@ extern "C" {
 q8_status q8_tune_gemm_tile(int block_n, int ctas);
 
 /* Tuning / test hook: epilogue warps per CTA of the cta_group::2 kernel for later calls in this process:
- * 8 (each warp walks four 32-column blocks per tile), 16 (two blocks per warp, both read out of the
- * accumulator before any arithmetic) or 0 = automatic.  Other values are Q8_ERR_ARG.  Results do not depend on it. */
+ * 8 (each warp walks four 32-column blocks per tile), 16 (two blocks per warp) or 0 = automatic.  Other values are Q8_ERR_ARG.  Results do not depend on it. */
 q8_status q8_tune_gemm_epilogue_warps(int warps);
 
 /* Tuning / test hook for the schedule of the cta_group::2 kernel.  When the number of 256 x 256 tiles

@@ -53,10 +53,7 @@ __device__ __forceinline__ void gelu_fast_x2(uint64_t y2, float &out_lo, float &
 // (row = lane, 16-byte piece g at position g ^ (lane & 7): bank-conflict free) and written by one
 // TMA store, clipped at the matrix edge by the hardware; otherwise every lane stores its own row.
 // Once the last TMEM load of the tile has landed the accumulator buffer is handed back (release()).
-// EAGER: all of the warp's TMEM loads are issued first and the accumulator is handed back before any arithmetic
-// (for kernels with a single accumulator buffer, where the tensor pipe idles until the buffer has been read out);
-// otherwise block by block, which needs 32 instead of COLS live accumulator registers.
-template <int COLS, bool EAGER = false, typename Release>
+template <int COLS, typename Release>
 __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
                                               const CUtensorMap *tmap_yq, bool yq_tma, uint32_t taddr, int64_t row0,
                                               int64_t col0, const int32_t (&bqv)[COLS / 32], const float (&invv)[COLS / 32],
@@ -183,25 +180,14 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
         }
     };
 
-    if constexpr (EAGER) {
-        uint32_t v[NCHUNK][32];
 #pragma unroll
-        for (int ci = 0; ci < NCHUNK; ++ci) tmem_ld_32x32(taddr + (uint32_t)(32 * ci), v[ci]);
+    for (int ci = 0; ci < NCHUNK; ++ci) {
+        if (ci >= nch) break;
+        uint32_t v[32];
+        tmem_ld_32x32(taddr + (uint32_t)(32 * ci), v);
         tmem_ld_wait();
-        release();
-#pragma unroll
-        for (int ci = 0; ci < NCHUNK; ++ci)
-            if (ci < nch) finish_block(v[ci], ci);
-    } else {
-#pragma unroll
-        for (int ci = 0; ci < NCHUNK; ++ci) {
-            if (ci >= nch) break;
-            uint32_t v[32];
-            tmem_ld_32x32(taddr + (uint32_t)(32 * ci), v);
-            tmem_ld_wait();
-            if (ci + 1 == nch) release();
-            finish_block(v, ci);
-        }
+        if (ci + 1 == nch) release();
+        finish_block(v, ci);
     }
     if (yq_pending) {
         // blocks beyond column N were never staged; the store clips them (and rows past M) at the matrix edge

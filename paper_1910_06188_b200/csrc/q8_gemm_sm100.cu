@@ -40,15 +40,7 @@ constexpr int kAccStages = 2;      // TMEM accumulator double buffering
 template <int BLOCK_N, int CTAS, int EW>
 struct Cfg {
     static constexpr int kEpilogueWarps = EW;
-    // With 16 epilogue warps the roles are aligned to warpgroups (warps 0..3: producer, MMA issuer, two idle warps;
-    // warps 4..19: epilogue) so that setmaxnreg can move registers from the issuing warpgroup to the epilogue warps:
-    // these then hold their whole 32 x 64 accumulator share at once and hand the TMEM buffer back before any arithmetic.
-    static constexpr bool kRegSplit = EW == 16;
-    static constexpr int kFirstEpilogueWarp = kRegSplit ? 4 : 2;
-    static constexpr int kThreads = 32 * (kFirstEpilogueWarp + EW);
-    static constexpr int kRegsIssue = 32, kRegsEpilogue = 112, kRegsAtLaunch = 96;
-    static_assert(!kRegSplit || 128 * kRegsIssue + 32 * EW * kRegsEpilogue <= kThreads * kRegsAtLaunch,
-                  "setmaxnreg split exceeds the registers of the launch");
+    static constexpr int kThreads = 64 + 32 * EW;
     static constexpr int kBRows = BLOCK_N / CTAS;  // W_q rows each CTA loads
     static constexpr int kABytes = BLOCK_M * BLOCK_K;
     static constexpr int kBBytes = kBRows * BLOCK_K;
@@ -75,7 +67,7 @@ struct Cfg {
 
 // ------------------------------------------------------------------ the kernel
 template <int BLOCK_N, int CTAS, int EW>
-__global__ void __launch_bounds__(Cfg<BLOCK_N, CTAS, EW>::kThreads, 1)
+__global__ void __launch_bounds__(64 + 32 * EW, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_w4,
                     const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_yq, GemmArgs a,
@@ -149,9 +141,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // produced X_q) must be complete before anything below reads global memory
     grid_dependency_wait();
 
-    // Each role's code sits in the same branch as its register-count change, so that it is compiled for that count.
-    if (warp < C::kFirstEpilogueWarp) {
-    if (C::kRegSplit) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsIssue));
     if (warp == 0) {
         // ---------------- TMA producer (each CTA loads its own rows) ----------------
         if (lane == 0) {
@@ -255,11 +244,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                        global_timer_ns() - t0 < 50000000ull) {}
             }
         }
-    }
     } else {
         // ---------------- epilogue ----------------
-        if (C::kRegSplit) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsEpilogue));
-        const int ew = warp - C::kFirstEpilogueWarp;  // 0 .. EW-1
+        const int ew = warp - 2;       // 0 .. EW-1
         const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32*quarter .. +31
         const int col_group = ew >> 2;  // which share of the tile's columns this warp takes
         const float S_x = __ldg(a.S_x);
@@ -326,7 +313,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
             };
             if (active)
-                epilogue_warp<C::kColsPerWarp, C::kRegSplit>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
+                epilogue_warp<C::kColsPerWarp>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                                                m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release,
                                                absmax_run);
@@ -371,14 +358,6 @@ cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
-        if (C::kRegSplit) {
-            // setmaxnreg.inc draws on the registers the block was launched with; a launch with fewer registers per
-            // thread than the split assumes would wait forever, so refuse it here
-            cudaFuncAttributes fa;
-            e = cudaFuncGetAttributes(&fa, kernel);
-            if (e != cudaSuccess) return e;
-            if (fa.numRegs < C::kRegsAtLaunch) return cudaErrorLaunchOutOfResources;
-        }
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         int units = sm_count() / CTAS;

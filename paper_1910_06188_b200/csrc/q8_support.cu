@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(kLnThreads) add_layernorm_vec_kernel(const flo
 
 // One warp per row for H <= 1024 (BERT's hidden sizes): up to eight float4 per lane, both moments reduced with
 // shuffles only, eight rows per CTA, so there is no block-level barrier at all.
-__global__ void __launch_bounds__(kLnThreads) add_layernorm_warp_kernel(const float *__restrict__ x,
+__global__ void __launch_bounds__(kLnThreads, kLnCtasPerSm) add_layernorm_warp_kernel(const float *__restrict__ x,
                                                                         const float *__restrict__ r1,
                                                                         const float *__restrict__ r2,
                                                                         const float *__restrict__ gamma,
