@@ -40,7 +40,7 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of the tcgen05 GEMM per launch on the BERT-Large FC set, from the
 # ncu captures summarised in profiles/gemm_tcgen05_dram_traffic_m24576.md (one layer resident per capture).  Below the
 # algorithmic bytes because part of each output is still dirty in the 126 MB L2 when the kernel ends.
-GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 270513664, "attn_out": 67436288, "ffn1": 372471296, "ffn2": 164332800}}
+GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 269627136, "attn_out": 66861568, "ffn1": 371578880, "ffn2": 163783168}}
 NOMINAL_INT8_OVER_BF16 = 2.0  # dense tensor peak ratio int8 : bf16 (4.5 : 2.25 POPS nominal)
 GEMM_REPS = 4   # launches per event pair in the per-kernel pass
 QUANT_REPS = 4  # times each group of equal-sized quantise passes is repeated per event pair
@@ -890,6 +890,19 @@ def measure_encoders(args, torch, q8):
         torch.cuda.synchronize()
         ms_graph = e0.elapsed_time(e1) / reps
         del graph
+        # dynamic quantisation (Sec. 4.1): every FC computing its own max|x|, against producers folding it
+        dyn = {}
+        for label, run in (("dynamic", lambda: enc.forward(ids, B, S, scales="dynamic")),
+                           ("dynamic_fused_absmax", lambda: enc.forward_dynamic_fused(ids, B, S))):
+            for _ in range(2):
+                run()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(reps):
+                run()
+            e1.record()
+            torch.cuda.synchronize()
+            dyn[label] = e0.elapsed_time(e1) / reps
         codes = enc.poll()
         # breakdown: time the three kinds of calls of one forward
         shares = {"q8_linear": 0.0, "attention_fp32": 0.0, "layernorm_embedding": 0.0}
@@ -943,6 +956,8 @@ def measure_encoders(args, torch, q8):
             "tokens_per_s": T / (ms * 1e-3), "ms_per_forward": ms, "layers": enc.L, "tokens": T,
             "tokens_per_s_fused_requant": T / (ms_fused * 1e-3), "ms_per_forward_fused_requant": ms_fused,
             "tokens_per_s_fused_cuda_graph": T / (ms_graph * 1e-3), "ms_per_forward_fused_cuda_graph": ms_graph,
+            "ms_per_forward_dynamic": dyn["dynamic"], "ms_per_forward_dynamic_fused_absmax": dyn["dynamic_fused_absmax"],
+            "tokens_per_s_dynamic_fused_absmax": T / (dyn["dynamic_fused_absmax"] * 1e-3),
             "gpu_launches_per_forward": enc.launches_per_forward(),
             "gpu_launches_per_forward_fused_requant": enc.launches_per_forward(fused=True),
             "status": [list(c) for c in codes],

@@ -22,6 +22,9 @@
  *     selects the vectorised / tensor-core kernels, anything else runs the generic kernels
  *     with identical results.
  *   - Results are deterministic: the same inputs give bit-identical outputs.
+ *
+ * Tuning hooks, measurement aids and the wait self-test live in q8_tools.h (same library); nothing in this header
+ * depends on them.
  */
 #ifndef Q8_H_
 #define Q8_H_

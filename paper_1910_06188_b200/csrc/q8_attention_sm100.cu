@@ -115,7 +115,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
 
     if (tid == 0) {
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&ready_bar[b]), kWorkers);
+            mbar_init(smem_u32(&ready_bar[b]), kWorkers / 32);  // one arrival per worker warp
             mbar_init(smem_u32(&done_bar[b]), 1);
         }
         abort_flag = 0;
@@ -130,14 +130,17 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
     grid_dependency_wait();  // the set-up above may overlap the tail of the kernel that produced qkv
 
     if (warp == kWorkers / 32) {
-        // ================= MMA warp: one lane issues, chunk after chunk, as the workers report operands ready
-        if (lane == 0) {
+        // ================= MMA warp: stays converged (all lanes wait and compute the same descriptors, which the
+        // compiler can then keep in uniform registers); one elected lane issues, chunk after chunk, as the workers
+        // report operands ready
+        {
+            const uint32_t elected = elect_one();
             uint32_t ready_phase = 0u;  // bit b: parity of the next phase of ready_bar[b]
             bool ok = true;
             const uint32_t q_hi = smem_u32(q_buf), q_lo = q_hi + 2 * kSpanBytesA;
             for (int kc = 0; kc < big_chunks && ok; ++kc) {  // scores of the 128 keys of big chunk kc
                 const int b = kc & 1;
-                ok = mbar_wait(smem_u32(&ready_bar[b]), (ready_phase >> b) & 1u, &abort_flag, status);
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&ready_bar[b]), (ready_phase >> b) & 1u, &abort_flag, status));
                 ready_phase ^= 1u << b;
                 if (!ok) break;
                 tc_fence_after();
@@ -150,17 +153,17 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {  // 8 fp32 = 32 bytes of K per instruction: +2 in the (address >> 4) field
                         const uint64_t adv = (uint64_t)(2 * ks);
-                        umma_tf32(d, al + adv, bh + adv, kIdescN128, acc);  // small terms first
-                        umma_tf32(d, ah + adv, bl + adv, kIdescN128, 1u);
-                        umma_tf32(d, ah + adv, bh + adv, kIdescN128, 1u);
+                        umma_tf32_elected(elected, d, al + adv, bh + adv, kIdescN128, acc);  // small terms first
+                        umma_tf32_elected(elected, d, ah + adv, bl + adv, kIdescN128, 1u);
+                        umma_tf32_elected(elected, d, ah + adv, bh + adv, kIdescN128, 1u);
                         acc = 1u;
                     }
                 }
-                umma_commit(smem_u32(&done_bar[b]));
+                umma_commit_elected(elected, smem_u32(&done_bar[b]));
             }
             for (int kc = 0; kc < chunks && ok; ++kc) {  // O += P V of chunk kc
                 const int b = kc & 1;
-                ok = mbar_wait(smem_u32(&ready_bar[b]), (ready_phase >> b) & 1u, &abort_flag, status);
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&ready_bar[b]), (ready_phase >> b) & 1u, &abort_flag, status));
                 ready_phase ^= 1u << b;
                 if (!ok) break;
                 tc_fence_after();
@@ -173,12 +176,12 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint64_t adv = (uint64_t)(2 * ks);
-                        umma_tf32(tmem_o, ah + adv, bhl + adv, kIdescN128, acc);         // [P_hi V_hi | P_hi V_lo]
-                        umma_tf32(tmem_o + kHeadDim, al + adv, bhl + adv, kIdescN64, 1u);  // += P_lo V_hi
+                        umma_tf32_elected(elected, tmem_o, ah + adv, bhl + adv, kIdescN128, acc);         // [P_hi V_hi | P_hi V_lo]
+                        umma_tf32_elected(elected, tmem_o + kHeadDim, al + adv, bhl + adv, kIdescN64, 1u);  // += P_lo V_hi
                         acc = 1u;
                     }
                 }
-                umma_commit(smem_u32(&done_bar[b]));
+                umma_commit_elected(elected, smem_u32(&done_bar[b]));
             }
         }
     } else {
@@ -195,10 +198,12 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             ok = __all_sync(0xffffffffu, mine);
             tc_fence_after();
         };
-        // this thread's shared-memory writes become visible to the tensor core, then it reports in
+        // every thread makes its shared-memory writes visible to the tensor core; then one lane reports for the warp
+        // (16 arrivals on the barrier instead of 512)
         auto report_ready = [&](int b) {
             fence_proxy_async_smem();
-            mbar_arrive(smem_u32(&ready_bar[b]));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ready_bar[b]));
         };
 
         // ---------------- phase 1: scores = (Q * log2(e)/8) K^T
@@ -226,10 +231,11 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             }
         };
         float m = -INFINITY;
-        auto take_max = [&](int c) {  // this thread's 32 columns of big chunk c
-            uint32_t v[32];
+        uint32_t sv[32];  // this thread's 32 score columns of a big chunk, on their way out of TMEM
+        auto load_scores = [&](int c) { tmem_ld_32x32(t_row + (uint32_t)(c * kBigChunk + cq * 32), sv); };
+        auto take_max = [&](int c) {  // after load_scores(c): waits for the load, folds the 32 columns into m
+            uint32_t(&v)[32] = sv;
             const int col0 = c * kBigChunk + cq * 32;
-            tmem_ld_32x32(t_row + (uint32_t)col0, v);
             tmem_ld_wait();
             if (col0 + 32 <= S) {
 #pragma unroll
@@ -246,7 +252,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             if (kc >= 2) {  // buffer b was read by the MMAs of big chunk kc - 2, whose scores are final after this wait
                 wait_done(b);
                 if (!ok) break;
-                take_max(kc - 2);
+                load_scores(kc - 2);  // in flight while the next K chunk is staged below
             }
 #pragma unroll
             for (int i = 0; i < kPiecesK; ++i) {
@@ -256,10 +262,14 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             }
             if (kc + 1 < big_chunks) fetch_k((kc + 1) * kBigChunk);  // next K chunk, in flight during the MMAs
             report_ready(b);
+            if (kc >= 2) take_max(kc - 2);
         }
         for (int c = (big_chunks > 2 ? big_chunks - 2 : 0); c < big_chunks && ok; ++c) {  // the last two big chunks
             wait_done(c & 1);
-            if (ok) take_max(c);
+            if (ok) {
+                load_scores(c);
+                take_max(c);
+            }
         }
         row_part[cq][row] = m;
         worker_barrier();
@@ -281,8 +291,26 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             }
         };
         if (ok) fetch_v(0);
+        // All scores are final, so a chunk's 16 score columns are fetched from TMEM one chunk ahead, and its
+        // exponentials are taken before the wait for the buffer set they will be stored into.
+        uint32_t pv[16];
+        if (ok) tmem_ld_32x16(t_row + (uint32_t)(cq * 16), pv);
         for (int kc = 0; kc < chunks && ok; ++kc) {
             const int b = kc & 1;
+            float p[16];
+            {
+                const int col0 = kc * kChunk + cq * 16;
+                tmem_ld_wait();
+                const bool whole = col0 + 16 <= S;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    float e;
+                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(__uint_as_float(pv[j]) - m));
+                    p[j] = (whole || col0 + j < S) ? e : 0.0f;
+                    l += p[j];
+                }
+                if (kc + 1 < chunks) tmem_ld_32x16(t_row + (uint32_t)(col0 + kChunk), pv);
+            }
             if (kc >= 2) {  // buffer set b was last read by the MMAs of chunk kc - 2
                 wait_done(b);
                 if (!ok) break;
@@ -297,19 +325,6 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             if (kc + 1 < chunks) fetch_v((kc + 1) * kChunk);
             // P[row][key]: this thread's 16 keys are pieces 4 (cq & 1) .. + 3 of span cq / 2 of the chunk
             {
-                uint32_t v[16];
-                const int col0 = kc * kChunk + cq * 16;
-                tmem_ld_32x16(t_row + (uint32_t)col0, v);
-                tmem_ld_wait();
-                float p[16];
-                const bool whole = col0 + 16 <= S;
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float e;
-                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(__uint_as_float(v[j]) - m));
-                    p[j] = (whole || col0 + j < S) ? e : 0.0f;
-                    l += p[j];
-                }
                 uint8_t *sb = p_buf(b) + (cq >> 1) * kSpanBytesA;
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
@@ -319,6 +334,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             }
             report_ready(b);
         }
+        tmem_ld_wait();  // (a load is still in flight only when the loop above was left early)
         for (int c = (chunks > 2 ? chunks - 2 : 0); c < chunks && ok; ++c) wait_done(c & 1);  // the last two chunks
 
         // ---------------- phase 3: ctx = (O_main + O_corr) / row sum
