@@ -243,6 +243,11 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     launches_per_step = 0
+    profile_S_y = None
+    if args.profile_mode and args.profile_int8_out:
+        profile_S_y = torch.full((1,), 20.0, device=dev)
+        for L in layers:
+            L["Yq_prof"] = torch.empty((L["M"], L["N"]), dtype=torch.int8, device=dev)
 
     # The four FC layers of the set (and the embedding gather) are independent of one another, so with
     # --streams > 1 each runs on its own stream: the HBM-bound quantise / gather passes of one layer overlap the
@@ -258,6 +263,11 @@ def run_ours(args):
         n = 0
         work = [lambda: q8.q8_embedding(ids, Eq, S_e, out=emb_out)]
         for L in layers:
+            if args.profile_mode and args.profile_int8_out:
+                # for ncu captures of the re-quantising epilogue: the layer emits only Int8, at a fixed scale
+                work.append(lambda L=L: q8.q8_linear_requant(L["Xd"], L["Wq"], L["S_w"], L["S_x"], L["bd"], L["act"],
+                                                             profile_S_y, Yq=L["Yq_prof"], workspace=L["ws"]))
+                continue
             work.append(lambda L=L: q8.q8_linear(L["Xd"], L["Wq"], L["S_w"], L["S_x"], L["bd"], L["act"], Y=L["Y"],
                                                  workspace=L["ws"]))
         if not side:
@@ -422,22 +432,8 @@ def run_ours(args):
                 print(f"[bench] CUDA graph capture of the per-kernel pass failed ({ex}); timing eager launches", file=sys.stderr)
                 gemm_graphs, quant_graphs, emb_graph, i8_graph, emb_cold_graph = [], {}, None, None, None
         for _ in range(ksteps):
-            ev_e0.record(stream)
-            if emb_graph is not None:
-                emb_graph.replay()
-            else:
-                for r in range(EMB_REPS):
-                    q8.q8_embedding(ids, Eq, S_e, out=emb_out if r % 2 == 0 else emb_out2)
-            ev_e1.record(stream)
-            for k, members in groups.items():
-                gev[k][0].record(stream)
-                if k in quant_graphs:
-                    quant_graphs[k].replay()
-                else:
-                    for _ in range(QUANT_REPS):
-                        for i in members:
-                            q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
-                gev[k][1].record(stream)
+            # the GEMMs first (right after the synchronisation below, i.e. from the same state as in a step), then the
+            # HBM-bound passes
             for i, L in enumerate(layers):
                 evs[i][1].record(stream)
                 if gemm_graphs:
@@ -453,6 +449,22 @@ def run_ours(args):
                 else:
                     run_i8()
                 ev_i1.record(stream)
+            for k, members in groups.items():
+                gev[k][0].record(stream)
+                if k in quant_graphs:
+                    quant_graphs[k].replay()
+                else:
+                    for _ in range(QUANT_REPS):
+                        for i in members:
+                            q8.q8_quantize_activation(layers[i]["Xd"], layers[i]["S_x"], Xq=layers[i]["Xq"])
+                gev[k][1].record(stream)
+            ev_e0.record(stream)
+            if emb_graph is not None:
+                emb_graph.replay()
+            else:
+                for r in range(EMB_REPS):
+                    q8.q8_embedding(ids, Eq, S_e, out=emb_out if r % 2 == 0 else emb_out2)
+            ev_e1.record(stream)
             ev_c0.record(stream)
             if emb_cold_graph is not None:
                 emb_cold_graph.replay()
@@ -995,6 +1007,8 @@ def main():
                     help="only warm-up + timed steps (no per-kernel pass, e2e or CPU baseline): for ncu captures")
     ap.add_argument("--encoder-kernel", choices=["attention", "layernorm"], default="",
                     help="with --profile-mode: launch only this FP32 support kernel of the encoder (--steps times)")
+    ap.add_argument("--profile-int8-out", action="store_true",
+                    help="with --profile-mode: the FC layers emit only Int8 (q8_linear_requant), for captures of that epilogue")
     ap.add_argument("--profile-batch", type=int, default=8)
     ap.add_argument("--profile-seq", type=int, default=384)
     ap.add_argument("--profile-heads", type=int, default=16)

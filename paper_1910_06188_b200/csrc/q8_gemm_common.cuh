@@ -53,7 +53,9 @@ __device__ __forceinline__ void gelu_fast_x2(uint64_t y2, float &out_lo, float &
 // (row = lane, 16-byte piece g at position g ^ (lane & 7): bank-conflict free) and written by one
 // TMA store, clipped at the matrix edge by the hardware; otherwise every lane stores its own row.
 // Once the last TMEM load of the tile has landed the accumulator buffer is handed back (release()).
-template <int COLS, typename Release>
+// ABSMAX: also keep the running max|y| of what is stored (a compile-time switch, so that the ordinary layer carries
+// neither the extra register nor the branch).
+template <int COLS, bool ABSMAX, typename Release>
 __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
                                               const CUtensorMap *tmap_yq, bool yq_tma, uint32_t taddr, int64_t row0,
                                               int64_t col0, const int32_t (&bqv)[COLS / 32], const float (&invv)[COLS / 32],
@@ -111,7 +113,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__fmul_rn(__int2float_rn((int32_t)v[j]), inv));
         }
-        if (a.y_absmax != nullptr && row_ok) {
+        if (ABSMAX && row_ok) {
             // running max|y| of this lane over the outputs that exist (Sec. 4.1: the consumer's dynamic scale)
             const bool whole = nb + 32 <= a.N;
 #pragma unroll

@@ -66,7 +66,7 @@ struct Cfg {
 };
 
 // ------------------------------------------------------------------ the kernel
-template <int BLOCK_N, int CTAS, int EW>
+template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_w4,
@@ -143,7 +143,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     if (warp == 0) {
         // ---------------- TMA producer (each CTA loads its own rows) ----------------
-        if (lane == 0) {
+        // (a converged warp with one elected issuing lane, like the MMA warp below)
+        {
+            const uint32_t elected = elect_one();
             int s = 0;
             uint32_t phase = 0;
             int issued = 0;
@@ -158,20 +160,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 const CUtensorMap *map_w = width == BLOCK_N ? &tmap_w : (width * 2 == BLOCK_N ? &tmap_w2 : &tmap_w4);
                 const uint32_t stage_bytes = (uint32_t)(C::kABytes + b_rows * BLOCK_K);
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = mbar_wait(smem_u32(empty_bar + s), phase ^ 1u, abort_flag, a.status);
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(empty_bar + s), phase ^ 1u, abort_flag, a.status));
                     if (!ok) break;
                     const uint32_t fb = smem_u32(full_bar + s);
                     const uint32_t dst_a = smem_u32(smem_a + s * C::kABytes), dst_b = smem_u32(smem_b + s * C::kBBytes);
                     if (CTAS == 1) {
-                        mbar_expect_tx(fb, stage_bytes);
-                        tma_load_2d(dst_a, &tmap_x, kb * BLOCK_K, m0, fb);
-                        tma_load_2d(dst_b, map_w, kb * BLOCK_K, n0, fb);
+                        mbar_expect_tx_elected(elected, fb, stage_bytes);
+                        tma_load_2d_elected(elected, dst_a, &tmap_x, kb * BLOCK_K, m0, fb);
+                        tma_load_2d_elected(elected, dst_b, map_w, kb * BLOCK_K, n0, fb);
                     } else {
                         // both CTAs report their bytes to the leader's barrier, which the MMA warp waits on
-                        if (leader) mbar_expect_tx(fb, 2 * stage_bytes);
+                        if (leader) mbar_expect_tx_elected(elected, fb, 2 * stage_bytes);
                         const uint32_t fb_leader = map_to_cta(fb, 0);
-                        tma_load_2d_pair(dst_a, &tmap_x, kb * BLOCK_K, m0, fb_leader);
-                        tma_load_2d_pair(dst_b, map_w, kb * BLOCK_K, n0, fb_leader);
+                        tma_load_2d_pair_elected(elected, dst_a, &tmap_x, kb * BLOCK_K, m0, fb_leader);
+                        tma_load_2d_pair_elected(elected, dst_b, map_w, kb * BLOCK_K, n0, fb_leader);
                     }
                     ++issued;
                     if (++s == C::kStages) { s = 0; phase ^= 1u; }
@@ -195,7 +197,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (the leader CTA drives the pair) ----------------
-        if (lane == 0 && leader) {
+        // The warp stays converged: every lane waits and computes the same descriptors (which the compiler can then
+        // hold in uniform registers, where tcgen05.mma wants them) and one elected lane issues the tensor-core
+        // instructions.  Against a single active lane: FFN2 (K = 4096, issue-rate sensitive) 80.3 -> 77.2 us, the
+        // other shapes 0-3 % faster.
+        if (leader) {
+            const uint32_t elected = elect_one();
+            auto uniform = [&](bool mine) { return (bool)__all_sync(0xffffffffu, mine); };
             int s = 0;
             uint32_t phase = 0;
             int as = 0;
@@ -204,7 +212,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             int last_as = 0;
             uint32_t last_aphase = 0;
             for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
-                ok = mbar_wait(smem_u32(tmem_empty_bar + as), aphase ^ 1u, abort_flag, a.status);
+                ok = uniform(mbar_wait(smem_u32(tmem_empty_bar + as), aphase ^ 1u, abort_flag, a.status));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(as * BLOCK_N);
@@ -212,7 +220,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 const uint32_t width = tile < full_tiles ? (uint32_t)BLOCK_N : (uint32_t)(BLOCK_N / split);
                 const uint32_t idesc = (C::kInstrDesc & ~(0x3Fu << 17)) | ((width >> 3) << 17);
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = mbar_wait(smem_u32(full_bar + s), phase, abort_flag, a.status);
+                    ok = uniform(mbar_wait(smem_u32(full_bar + s), phase, abort_flag, a.status));
                     if (!ok) break;
                     tc_fence_after();
                     const uint64_t da = smem_desc_sw128(smem_u32(smem_a + s * C::kABytes));
@@ -221,17 +229,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                         // +32 bytes along K inside the swizzle span == +2 in the (addr >> 4) field
                         const uint64_t adv = (uint64_t)(k * (UMMA_K >> 4));
-                        if (CTAS == 2) umma_i8_pair(tmem_d, da + adv, db + adv, idesc, (uint32_t)((kb | k) != 0));
-                        else umma_i8(tmem_d, da + adv, db + adv, idesc, (uint32_t)((kb | k) != 0));
+                        if (CTAS == 2) umma_i8_pair_elected(elected, tmem_d, da + adv, db + adv, idesc, (uint32_t)((kb | k) != 0));
+                        else umma_i8_elected(elected, tmem_d, da + adv, db + adv, idesc, (uint32_t)((kb | k) != 0));
                     }
                     // frees the stage (in both CTAs) once these MMAs have read it
-                    if (CTAS == 2) umma_commit_pair(smem_u32(empty_bar + s));
-                    else umma_commit(smem_u32(empty_bar + s));
+                    if (CTAS == 2) umma_commit_pair_elected(elected, smem_u32(empty_bar + s));
+                    else umma_commit_elected(elected, smem_u32(empty_bar + s));
                     if (++s == C::kStages) { s = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                if (CTAS == 2) umma_commit_pair(smem_u32(tmem_full_bar + as));  // accumulator complete
-                else umma_commit(smem_u32(tmem_full_bar + as));
+                if (CTAS == 2) umma_commit_pair_elected(elected, smem_u32(tmem_full_bar + as));  // accumulator complete
+                else umma_commit_elected(elected, smem_u32(tmem_full_bar + as));
                 committed = true;
                 last_as = as;
                 last_aphase = aphase;
@@ -313,7 +321,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
             };
             if (active)
-                epilogue_warp<C::kColsPerWarp>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
+                epilogue_warp<C::kColsPerWarp, ABSMAX>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                                                m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release,
                                                absmax_run);
@@ -321,7 +329,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 release();
             if (++as == kAccStages) { as = 0; aphase ^= 1u; }
         }
-        if (a.y_absmax != nullptr) warp_fold_absmax(absmax_run, a.y_absmax);  // one atomic per epilogue warp and launch
+        if (ABSMAX) warp_fold_absmax(absmax_run, a.y_absmax);  // one atomic per epilogue warp and launch
         if (lane == 0) tma_store_wait_all();
     }
 
@@ -345,12 +353,23 @@ int g_force_block_n = 0, g_force_ctas = 0;  // set by q8_tune_gemm_tile(); 0 = c
 int g_force_epilogue_warps = 0;            // 0 automatic, else 8 or 16 (cta_group::2 kernel only)
 bool g_tail_split_enabled = true;          // cut the tiles of a partial last round into narrower ones
 
+template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
+cudaError_t launch_cfg_impl(const GemmArgs &a, cudaStream_t s);
+
+// The layer that also reports max|y| (Sec. 4.1 chained dynamically) runs its own instantiation of the kernel.
 template <int BLOCK_N, int CTAS, int EW = 8>
 cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
 {
+    return a.y_absmax != nullptr ? launch_cfg_impl<BLOCK_N, CTAS, EW, true>(a, s)
+                                 : launch_cfg_impl<BLOCK_N, CTAS, EW, false>(a, s);
+}
+
+template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
+cudaError_t launch_cfg_impl(const GemmArgs &a, cudaStream_t s)
+{
     using C = Cfg<BLOCK_N, CTAS, EW>;
     constexpr int kThreads = C::kThreads;
-    auto kernel = gemm_tcgen05_kernel<BLOCK_N, CTAS, EW>;
+    auto kernel = gemm_tcgen05_kernel<BLOCK_N, CTAS, EW, ABSMAX>;
     static bool attr_set[64] = {};  // the opt-in shared-memory size is a per-device, per-function attribute
     static int max_units[64] = {};  // co-resident CTAs (CTAS = 1) or CTA pairs (CTAS = 2) on the device
     int dev = 0;
