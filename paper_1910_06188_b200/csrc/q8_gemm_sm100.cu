@@ -321,7 +321,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 }
             };
             if (active)
-                epilogue_warp<C::kColsPerWarp, ABSMAX>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
+                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8)>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                                                m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release,
                                                absmax_run);
