@@ -207,6 +207,17 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
         };
 
         // ---------------- phase 1: scores = (Q * log2(e)/8) K^T
+        constexpr int kPiecesK = (kBigChunk * 16) / kWorkers;  // 16-byte pieces of a 128-key K chunk per thread
+        float4 kreg[kPiecesK];
+        auto fetch_k = [&](int j0) {  // 128 keys x 64 fp32
+#pragma unroll
+            for (int i = 0; i < kPiecesK; ++i) {
+                const int c = tid + i * kWorkers, r = c >> 4, pc = c & 15;
+                kreg[i] = (j0 + r < S) ? __ldg(reinterpret_cast<const float4 *>(base + (int64_t)(j0 + r) * row_pitch + H) + pc)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        };
+        fetch_k(0);  // the first K chunk travels while Q is split and staged
         // a 16-byte piece c of a [rows x 64] fp32 tile: row c / 16, span (c % 16) / 8, piece (c % 16) % 8
 #pragma unroll
         for (int i = 0; i < (kQTile * 16) / kWorkers; ++i) {
@@ -220,16 +231,6 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             uint8_t *at = q_buf + (pc >> 3) * kSpanBytesA + sw128_offset(r, pc & 7);
             store_split4(at, at + 2 * kSpanBytesA, v);
         }
-        constexpr int kPiecesK = (kBigChunk * 16) / kWorkers;  // 16-byte pieces of a 128-key K chunk per thread
-        float4 kreg[kPiecesK];
-        auto fetch_k = [&](int j0) {  // 128 keys x 64 fp32
-#pragma unroll
-            for (int i = 0; i < kPiecesK; ++i) {
-                const int c = tid + i * kWorkers, r = c >> 4, pc = c & 15;
-                kreg[i] = (j0 + r < S) ? __ldg(reinterpret_cast<const float4 *>(base + (int64_t)(j0 + r) * row_pitch + H) + pc)
-                                       : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        };
         float m = -INFINITY;
         uint32_t sv[32];  // this thread's 32 score columns of a big chunk, on their way out of TMEM
         auto load_scores = [&](int c) { tmem_ld_32x32(t_row + (uint32_t)(c * kBigChunk + cq * 32), sv); };
@@ -246,7 +247,6 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
                     if (col0 + j < S) m = fmaxf(m, __uint_as_float(v[j]));
             }
         };
-        fetch_k(0);
         for (int kc = 0; kc < big_chunks && ok; ++kc) {
             const int b = kc & 1;
             if (kc >= 2) {  // buffer b was read by the MMAs of big chunk kc - 2, whose scores are final after this wait
@@ -335,11 +335,11 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             report_ready(b);
         }
         tmem_ld_wait();  // (a load is still in flight only when the loop above was left early)
+        row_part[cq][row] = l;  // the row sums are exchanged while the last MMAs run
+        worker_barrier();
         for (int c = (chunks > 2 ? chunks - 2 : 0); c < chunks && ok; ++c) wait_done(c & 1);  // the last two chunks
 
         // ---------------- phase 3: ctx = (O_main + O_corr) / row sum
-        row_part[cq][row] = l;
-        worker_barrier();
         if (ok) {  // (warp-uniform: the TMEM loads below are warp-wide instructions, only the stores depend on the row)
             const float inv = 1.0f / ((row_part[0][row] + row_part[1][row]) + (row_part[2][row] + row_part[3][row]));
             uint32_t v[16], w[16];
