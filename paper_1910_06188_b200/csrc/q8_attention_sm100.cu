@@ -127,6 +127,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
     const uint32_t tmem_o = tmem_base + (uint32_t)s_pad;  // O_main: 64 columns behind the scores; O_corr: the next 64
+    grid_dependency_release_next(gridDim.x * gridDim.y * gridDim.z <= 600u);  // up to ~4 waves of CTAs count as small
     grid_dependency_wait();  // the set-up above may overlap the tail of the kernel that produced qkv
 
     if (warp == kWorkers / 32) {

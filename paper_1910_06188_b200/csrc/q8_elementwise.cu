@@ -109,6 +109,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const float *__restr
                                                             int32_t *__restrict__ status = nullptr,
                                                             int32_t *__restrict__ clear_word = nullptr)
 {
+    grid_dependency_release_next(n <= kSmallProblemElems);
     grid_dependency_wait();
     // first kernel of a static-scale q8_linear call: start the call's status word at zero
     if (clear_word != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *clear_word = 0;
@@ -187,6 +188,7 @@ __global__ void __launch_bounds__(kDqThreads) quantize_dynamic_cluster_kernel(co
                                                                               int8_t *__restrict__ xq,
                                                                               int8_t *__restrict__ xq_copy)
 {
+    grid_dependency_release_next(true);  // small by construction
     grid_dependency_wait();
     __shared__ float warp_max[kDqThreads / 32];
     __shared__ float cta_max, all_max;
@@ -298,6 +300,7 @@ __global__ void __launch_bounds__(kThreads) embedding_kernel(const int32_t *__re
                                                              float *__restrict__ out, int8_t *__restrict__ rows_q,
                                                              int32_t *__restrict__ status)
 {
+    grid_dependency_release_next(T * H <= kSmallProblemElems);
     grid_dependency_wait();
     const float inv = __fdiv_rn(1.0f, __ldg(S_e));
     if (VEC) {

@@ -139,6 +139,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     const uint32_t tmem_base = *tmem_slot;
     // everything above touched only this CTA's own resources; the kernel before this one in the stream (which
     // produced X_q) must be complete before anything below reads global memory
+    grid_dependency_release_next(num_tiles <= 3 * num_units);  // up to three rounds of tiles count as small
     grid_dependency_wait();
 
     if (warp == 0) {

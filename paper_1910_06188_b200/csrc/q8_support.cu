@@ -141,6 +141,7 @@ __global__ void __launch_bounds__(kLnThreads, kLnCtasPerSm) add_layernorm_warp_k
                                                                         const float *__restrict__ S_q,
                                                                         int8_t *__restrict__ out_q, uint32_t *__restrict__ amax)
 {
+    grid_dependency_release_next(rows * H <= kSmallProblemElems);
     grid_dependency_wait();  // launched so that its start may overlap the tail of the kernel before it
     const int lane = threadIdx.x & 31;
     const int n4 = (int)(H >> 2);
