@@ -31,6 +31,12 @@ q8_status q8_tune_gemm_epilogue_warps(int warps);
  * not depend on it.  Not thread-safe.  (An implementation detail with no counterpart in the paper.) */
 void q8_tune_gemm_tail_split(int enable);
 
+/* Tuning / test hook for the way the tcgen05 GEMM writes a plain fp32 output (no Int8 copy asked for).
+ * mode 1: each epilogue warp reads its accumulator block in the 16 x 256 bit fragment layout and stores it
+ * straight from registers, every 32-byte sector written whole by four neighbouring lanes; mode 0: the block
+ * is staged in shared memory and leaves as a TMA store.  Results do not depend on it.  Not thread-safe. */
+void q8_tune_gemm_direct_store(int mode);
+
 /* Into how many narrower tiles each tile of the last round was cut by the most recent tcgen05 GEMM launch
  * of this host thread: 1 (not cut), 2 or 4. */
 int q8_last_launch_tail_split(void);

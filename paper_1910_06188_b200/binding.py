@@ -53,6 +53,7 @@ SIGNATURES = {
     "q8_last_launch_info": (None, [C.POINTER(_int)] * 5),
     "q8_tune_gemm_tile": (_int, [_int, _int]),
     "q8_tune_gemm_tail_split": (None, [_int]),
+    "q8_tune_gemm_direct_store": (None, [_int]),
     "q8_tune_attention": (None, [_int]),
     "q8_selftest_wait_timeout": (_int, [C.c_uint64, _vp, _vp, _vp]),
     "q8_attention_status_word": (_int, [C.POINTER(C.c_void_p)]),
@@ -545,6 +546,11 @@ def q8_tune_gemm_epilogue_warps(warps: int = 0) -> None:
 def q8_tune_gemm_tail_split(enable: bool = True) -> None:
     """Switches the cutting of the last scheduling round's tiles into narrower ones on or off."""
     load().q8_tune_gemm_tail_split(1 if enable else 0)
+
+
+def q8_tune_gemm_direct_store(mode: bool = True) -> None:
+    """fp32-only GEMM output stored straight from registers (True) or staged and TMA-stored (False)."""
+    load().q8_tune_gemm_direct_store(1 if mode else 0)
 
 
 def q8_last_launch_tail_split() -> int:

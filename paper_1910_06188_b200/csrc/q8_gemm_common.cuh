@@ -213,6 +213,88 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
     }
 }
 
+// The same work for the plain fp32 output (no Int8 copy), without the shared-memory staging: the accumulator block is
+// read in the 16x256b fragment layout, where four neighbouring lanes hold 32 contiguous bytes of a row, so each lane
+// stores its pairs straight to Y (8-byte stores, every sector written whole by one instruction).  No proxy fence,
+// no TMA store, no staging buffer to wait for.  Needs an even N and an 8-byte aligned Y.
+template <int COLS, bool ABSMAX, typename Release>
+__device__ __forceinline__ void epilogue_warp_direct(const GemmArgs &a, uint32_t taddr, int64_t row0, int64_t col0,
+                                                     const int32_t (&bqv)[COLS / 32], const float (&invv)[COLS / 32],
+                                                     int32_t *bq_s, int lane, int nch, Release release, float &absmax_run)
+{
+    constexpr int NCHUNK = COLS / 32;
+    const int g = lane >> 2, cq = 2 * (lane & 3);
+    uint32_t v[32];  // v[16 h + 4 i + 2 r + c]: row 16 h + 8 r + g, column 8 i + cq + c of the block
+#pragma unroll
+    for (int ci = 0; ci < NCHUNK; ++ci) {
+        if (ci >= nch) break;
+        tmem_ld_16x256b_x4(taddr + (uint32_t)(32 * ci), v);
+        tmem_ld_16x256b_x4(taddr + (16u << 16) + (uint32_t)(32 * ci), v + 16);
+        tmem_ld_wait();
+        if (ci + 1 == nch) release();
+        const int64_t nb = col0 + 32 * ci;
+        const float inv = invv[ci];
+        if (nb >= a.N || row0 >= a.M) continue;  // warp-uniform: the block lies outside the matrix
+        __syncwarp();
+        bq_s[lane] = bqv[ci];
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int2 b = *reinterpret_cast<const int2 *>(bq_s + 8 * i + cq);
+#pragma unroll
+            for (int hr = 0; hr < 4; ++hr) {
+                const int k = 16 * (hr >> 1) + 4 * i + 2 * (hr & 1);
+                v[k] = (uint32_t)add_wrap((int32_t)v[k], b.x);
+                v[k + 1] = (uint32_t)add_wrap((int32_t)v[k + 1], b.y);
+            }
+        }
+        if (a.dbg_acc != nullptr) {
+#pragma unroll
+            for (int hr = 0; hr < 4; ++hr) {
+                const int64_t row = row0 + 16 * (hr >> 1) + 8 * (hr & 1) + g;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int k = 16 * (hr >> 1) + 4 * i + 2 * (hr & 1);
+                    const int64_t col = nb + 8 * i + cq;
+                    if (row < a.M && col < a.N) {
+                        a.dbg_acc[row * a.N + col] = (int32_t)v[k];
+                        a.dbg_acc[row * a.N + col + 1] = (int32_t)v[k + 1];
+                    }
+                }
+            }
+        }
+        if (a.act == Q8_ACT_GELU) {
+            const uint64_t inv2 = pack_f32x2(inv, inv);
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                const uint64_t y2 =
+                    mul_f32x2(pack_f32x2(__int2float_rn((int32_t)v[j]), __int2float_rn((int32_t)v[j + 1])), inv2);
+                float g0, g1;
+                gelu_fast_x2(y2, g0, g1);
+                v[j] = __float_as_uint(g0);
+                v[j + 1] = __float_as_uint(g1);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__fmul_rn(__int2float_rn((int32_t)v[j]), inv));
+        }
+#pragma unroll
+        for (int hr = 0; hr < 4; ++hr) {
+            const int64_t row = row0 + 16 * (hr >> 1) + 8 * (hr & 1) + g;
+            float *yrow = a.Y + row * a.N + nb + cq;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int k = 16 * (hr >> 1) + 4 * i + 2 * (hr & 1);
+                if (row < a.M && nb + 8 * i + cq < a.N) {
+                    const float y0 = __uint_as_float(v[k]), y1 = __uint_as_float(v[k + 1]);
+                    if (ABSMAX) absmax_run = fmaxf(absmax_run, fmaxf(fabsf(y0), fabsf(y1)));
+                    *reinterpret_cast<float2 *>(yrow + 8 * i) = make_float2(y0, y1);
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,

@@ -101,16 +101,22 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     // BLOCK_N / split columns), so that the tail keeps more units busy for a shorter time.
     const int64_t num_tiles = full_tiles + (tiles_m * tiles_n - full_tiles) * split;
     const int32_t tiles_n32 = (int32_t)tiles_n, full32 = (int32_t)full_tiles;  // tile counts fit 32 bits by far
+    // Every warp decodes a tile index per tile, and in the epilogue warps that sits on the serial path between two
+    // accumulators, so it avoids integer division: split is 1, 2 or 4 (a shift), and whole / tiles_n is the high
+    // word of whole * ceil(2^32 / tiles_n), exact while whole * tiles_n < 2^32 (else the division is kept).
+    const int split_log2 = split >> 1;
+    const uint32_t tn_magic = 0xFFFFFFFFu / (uint32_t)tiles_n32 + 1u;
+    const bool tn_fast = tiles_n32 > 1 && (uint64_t)(tiles_m * tiles_n) * (uint64_t)tiles_n < (uint64_t(1) << 32);
     auto decode = [&](int64_t t, int64_t &m_idx, int64_t &n0, int &width) {
         int32_t whole = (int32_t)t, sub = 0;
         width = BLOCK_N;
         if (whole >= full32) {
             const int32_t u = whole - full32;
-            width = BLOCK_N / split;
-            whole = full32 + u / split;
-            sub = u % split;
+            width = BLOCK_N >> split_log2;
+            whole = full32 + (u >> split_log2);
+            sub = u & (split - 1);
         }
-        const int32_t mi = whole / tiles_n32;
+        const int32_t mi = tn_fast ? (int32_t)__umulhi((uint32_t)whole, tn_magic) : whole / tiles_n32;
         m_idx = mi;
         n0 = (whole - mi * tiles_n32) * BLOCK_N + sub * width;
     };
@@ -218,7 +224,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(as * BLOCK_N);
                 // a narrow tile of the split tail runs the same MMA with a smaller N field (bits 17..22 = N / 8)
-                const uint32_t width = tile < full_tiles ? (uint32_t)BLOCK_N : (uint32_t)(BLOCK_N / split);
+                const uint32_t width = tile < full_tiles ? (uint32_t)BLOCK_N : (uint32_t)(BLOCK_N >> split_log2);
                 const uint32_t idesc = (C::kInstrDesc & ~(0x3Fu << 17)) | ((width >> 3) << 17);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = uniform(mbar_wait(smem_u32(full_bar + s), phase, abort_flag, a.status));
@@ -291,6 +297,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             }
         };
         fetch_bias(unit, bias_next);
+        // one weight scale for the whole matrix (the usual case): the product scale and its reciprocal are
+        // computed once, not per tile (the load of S_w alone is a round trip to L2 under full operand traffic)
+        const bool one_scale = a.w_seg <= 0;
+        const float S_out_all = __fmul_rn(S_x, __ldg(a.S_w)), inv_all = __fdiv_rn(1.0f, S_out_all);
         for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
             int64_t m_idx, n0;
             int width;
@@ -303,26 +313,32 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             float invv[NCH];
 #pragma unroll
             for (int ci = 0; ci < NCH; ++ci) {
-                const float S_out = product_scale(n0 + col_off + 32 * ci);
+                const float S_out = one_scale ? S_out_all : product_scale(n0 + col_off + 32 * ci);
                 bqv[ci] = quantize_bias(bias_next[ci], S_out);
-                invv[ci] = __fdiv_rn(1.0f, S_out);
+                invv[ci] = one_scale ? inv_all : __fdiv_rn(1.0f, S_out);
             }
             fetch_bias(tile + num_units, bias_next);
             ok = mbar_wait(smem_u32(tmem_full_bar + as), aphase, abort_flag, a.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            // hands the accumulator buffer back to the MMA warp (called once this warp's TMEM loads are done)
+            // Hands the accumulator buffer back to the MMA warp (called once this warp's TMEM loads are done:
+            // tcgen05.wait::ld has returned in every lane, so the values are in registers).  The arrival carries no
+            // memory ordering: nothing this warp wrote to memory is read by the MMA warp.
             auto release = [&]() {
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    if (CTAS == 2) mbar_arrive_cluster(map_to_cta(smem_u32(tmem_empty_bar + as), 0));
+                    if (CTAS == 2) mbar_arrive_cluster_relaxed(map_to_cta(smem_u32(tmem_empty_bar + as), 0));
                     else mbar_arrive(smem_u32(tmem_empty_bar + as));
                 }
             };
-            if (active)
-                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8)>(a, &tmap_y, tma_store != 0, &tmap_yq, yq_tma != 0,
+            if (active && tma_store == 2)
+                epilogue_warp_direct<C::kColsPerWarp, ABSMAX>(
+                    a, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
+                    m0 + quarter * 32, n0 + col_off, bqv, invv, bq_s, lane, cpw / 32, release, absmax_run);
+            else if (active)
+                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8)>(a, &tmap_y, tma_store == 1, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                                                m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release,
                                                absmax_run);
@@ -352,6 +368,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 // ------------------------------------------------------------------ host side
 int g_force_block_n = 0, g_force_ctas = 0;  // set by q8_tune_gemm_tile(); 0 = choose automatically
 int g_force_epilogue_warps = 0;            // 0 automatic, else 8 or 16 (cta_group::2 kernel only)
+bool g_direct_store = false;               // fp32-only output stored from the 16x256b fragment layout, no staging
 bool g_tail_split_enabled = true;          // cut the tiles of a partial last round into narrower ones
 
 template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
@@ -425,7 +442,11 @@ cudaError_t launch_cfg_impl(const GemmArgs &a, cudaStream_t s)
     }
     // the TMA store needs a 16-byte aligned base and row pitch; otherwise lanes store their rows directly
     int tma_store = a.Y != nullptr && ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
-    if (tma_store) {
+    if (g_direct_store && a.Y != nullptr && a.Yq == nullptr && ((a.N & 1) == 0) &&
+        ((reinterpret_cast<uintptr_t>(a.Y) & 7u) == 0)) {
+        tma_store = 2;
+        ty = tx;
+    } else if (tma_store) {
         if (!make_tmap_out(&ty, a.Y, a.M, a.N)) return cudaErrorInvalidValue;
     } else {
         ty = tx;  // never dereferenced
@@ -496,6 +517,7 @@ void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps)
 }
 
 void set_gemm_tail_split(bool enable) { g_tail_split_enabled = enable; }
+void set_gemm_direct_store(bool enable) { g_direct_store = enable; }
 void set_gemm_epilogue_warps(int warps) { g_force_epilogue_warps = warps; }
 
 bool tcgen05_gemm_supported(const GemmArgs &a)

@@ -242,6 +242,19 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16])
         : "r"(taddr)
         : "memory");
 }
+// 16 lanes x 32 consecutive 32-bit columns in the 16x256b fragment layout: with g = lane / 4 and q = lane % 4,
+// r[4 i + 0 / 1] are columns 8 i + 2 q and 8 i + 2 q + 1 of TMEM lane g, r[4 i + 2 / 3] the same columns of lane
+// g + 8 (i = 0..3).  Four neighbouring lanes thus hold 32 contiguous bytes of one row: a whole memory sector.
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t *r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ---- cluster / cta_group::2 forms
@@ -265,6 +278,13 @@ __device__ __forceinline__ void cluster_sync_all()
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// The same arrival without memory ordering, for hand-overs that publish no memory: a cluster-scope release has to
+// wait for every memory access the thread still has in flight (a prefetched global load takes microseconds under
+// the main loop's operand traffic), which a pure "I am done reading TMEM" signal does not need.
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // Load into this CTA's shared memory; completion bytes are reported to an mbarrier that may live in
 // the other CTA of the pair (no multicast: every CTA fetches exactly the bytes it stores).
