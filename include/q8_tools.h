@@ -34,7 +34,9 @@ void q8_tune_gemm_tail_split(int enable);
 /* Tuning / test hook for the way the tcgen05 GEMM writes a plain fp32 output (no Int8 copy asked for).
  * mode 1: each epilogue warp reads its accumulator block in the 16 x 256 bit fragment layout and stores it
  * straight from registers, every 32-byte sector written whole by four neighbouring lanes; mode 0: the block
- * is staged in shared memory and leaves as a TMA store.  Results do not depend on it.  Not thread-safe. */
+ * is staged in shared memory and leaves as a TMA store; mode < 0 (the default): automatic, unstaged only for the
+ * CTA-pair kernel with the 8-warp epilogue (K > 2048), where it measured 2 % faster.  Results do not depend on
+ * it.  Not thread-safe. */
 void q8_tune_gemm_direct_store(int mode);
 
 /* Into how many narrower tiles each tile of the last round was cut by the most recent tcgen05 GEMM launch
@@ -67,6 +69,19 @@ q8_status q8_measure_int8_mma_peak(int ctas, double seconds, double *tops, doubl
  * Returns Q8_ERR_NULL / Q8_ERR_ALIGN / Q8_ERR_ARG (bytes < 16, repeats outside 1..1000) / Q8_ERR_CUDA. */
 q8_status q8_measure_hbm_peak(void *buf, size_t bytes, int store, int repeats, double *gbs, double *elapsed_ms,
                               void *stream);
+
+/* Measurement aid, no counterpart in the paper: the rate (GB/s, over all SMs) at which TMA pulls L2-resident
+ * operand boxes (128 rows x 128 bytes, the GEMM's operand box) into shared memory, with nothing else running:
+ * the ceiling of the GEMM's main loop when no operand byte is shared between SMs.  buf (device, 16-byte aligned)
+ * is read as a row-major Int8 matrix [rows, K] (rows % 128 == 0, K % 128 == 0; keep rows * K well below the L2
+ * size so that the timed launch reads from L2); every SM loads boxes_per_sm boxes through a ring of 12 stages.
+ * sms_used = 0 runs one CTA on every SM, a smaller positive number that many CTAs (to tell a per-SM limit from
+ * a limit of the L2 side).  producers = 1, 2, 3 or 4 warps issue the loads, each into its own share of the ring
+ * (one warp alone is bound by its own issue loop, about a box per 285 cycles).
+ * One untimed launch warms L2, the next is timed with CUDA events.  *gbs and *elapsed_ms (may be NULL) are host
+ * outputs.  Returns Q8_ERR_TIMEOUT if a bounded wait inside the kernel ran out.  Synchronises the stream. */
+q8_status q8_measure_l2_operand_peak(const void *buf, int64_t rows, int64_t K, int boxes_per_sm, int sms_used,
+                                     int producers, double *gbs, double *elapsed_ms, void *stream);
 
 /* Self-test of the bounded device-side wait every tensor-core kernel of the library is built on.  Launches one
  * small CTA that initialises an mbarrier nobody ever arrives on and waits on it with the library's own bounded

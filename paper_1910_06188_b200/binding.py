@@ -61,6 +61,8 @@ SIGNATURES = {
     "q8_last_launch_tail_split": (_int, []),
     "q8_measure_hbm_peak": (_int, [C.c_void_p, C.c_size_t, _int, _int, C.POINTER(C.c_double), C.POINTER(C.c_double),
                                    C.c_void_p]),
+    "q8_measure_l2_operand_peak": (_int, [C.c_void_p, C.c_int64, C.c_int64, _int, _int, _int, C.POINTER(C.c_double),
+                                          C.POINTER(C.c_double), C.c_void_p]),
     "q8_measure_int8_mma_peak": (_int, [_int, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(_int),
                                         C.c_void_p, C.c_void_p]),
 }
@@ -511,6 +513,19 @@ def q8_measure_hbm_peak(buf: torch.Tensor, store: bool, repeats: int = 10, strea
     return {"gbs": gbs.value, "elapsed_ms": ms.value, "bytes": nbytes, "repeats": int(repeats), "store": bool(store)}
 
 
+def q8_measure_l2_operand_peak(buf: torch.Tensor, rows: int, K: int, boxes_per_sm: int = 2048, sms_used: int = 0,
+                               producers: int = 4, stream=None) -> dict:
+    """Rate at which all SMs pull L2-resident 128 x 128-byte operand boxes of the Int8 matrix buf[rows, K] by TMA."""
+    gbs, ms = C.c_double(0.0), C.c_double(0.0)
+    if buf.numel() * buf.element_size() < rows * K:
+        raise ValueError("buf is smaller than rows * K bytes")
+    st = load().q8_measure_l2_operand_peak(_any_ptr(buf, "buf"), int(rows), int(K), int(boxes_per_sm), int(sms_used),
+                                           int(producers), C.byref(gbs), C.byref(ms), _stream(stream))
+    _check(st, "q8_measure_l2_operand_peak")
+    return {"gbs": gbs.value, "elapsed_ms": ms.value, "rows": int(rows), "K": int(K), "boxes_per_sm": int(boxes_per_sm),
+            "sms_used": int(sms_used), "producers": int(producers)}
+
+
 def q8_selftest_wait_timeout(limit_ns: int, dev_status: torch.Tensor, dev_report: Optional[torch.Tensor] = None,
                              stream=None) -> None:
     """Launches the library's wait self-test: one CTA waits (bounded by limit_ns) on a barrier nobody arrives on."""
@@ -548,9 +563,9 @@ def q8_tune_gemm_tail_split(enable: bool = True) -> None:
     load().q8_tune_gemm_tail_split(1 if enable else 0)
 
 
-def q8_tune_gemm_direct_store(mode: bool = True) -> None:
-    """fp32-only GEMM output stored straight from registers (True) or staged and TMA-stored (False)."""
-    load().q8_tune_gemm_direct_store(1 if mode else 0)
+def q8_tune_gemm_direct_store(mode: Optional[bool] = None) -> None:
+    """fp32-only GEMM output stored straight from registers (True), staged and TMA-stored (False) or automatic (None)."""
+    load().q8_tune_gemm_direct_store(-1 if mode is None else (1 if mode else 0))
 
 
 def q8_last_launch_tail_split() -> int:

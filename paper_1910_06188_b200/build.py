@@ -13,7 +13,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libq8.so")
 
-SOURCES = ["q8_api.cu", "q8_attention_sm100.cu", "q8_elementwise.cu", "q8_gemm_generic.cu", "q8_gemm_sm100.cu", "q8_hbm_peak.cu", "q8_mma_peak.cu", "q8_selftest.cu", "q8_static_scratch.cu", "q8_support.cu"]
+SOURCES = ["q8_api.cu", "q8_attention_sm100.cu", "q8_elementwise.cu", "q8_gemm_generic.cu", "q8_gemm_sm100.cu", "q8_hbm_peak.cu", "q8_l2_peak.cu", "q8_mma_peak.cu", "q8_selftest.cu", "q8_static_scratch.cu", "q8_support.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-O3", "-std=c++17", "-lineinfo",

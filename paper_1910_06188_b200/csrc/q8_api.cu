@@ -507,7 +507,7 @@ q8_status q8_attention_status_word(void **dev_status)
 }
 
 void q8_tune_gemm_tail_split(int enable) { set_gemm_tail_split(enable != 0); }
-void q8_tune_gemm_direct_store(int mode) { set_gemm_direct_store(mode != 0); }
+void q8_tune_gemm_direct_store(int mode) { set_gemm_direct_store(mode); }
 
 int q8_last_launch_tail_split(void) { return last_launch_info().tail_split; }
 

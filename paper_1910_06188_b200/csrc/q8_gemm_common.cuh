@@ -57,7 +57,9 @@ __device__ __forceinline__ void gelu_fast_x2(uint64_t y2, float &out_lo, float &
 // neither the extra register nor the branch).
 // PREFETCH: issue the next block's TMEM load before the proxy fence and TMA store of the current one (pays when a
 // warp walks four blocks per tile; with two blocks per warp it measured 1 % slower).
-template <int COLS, bool ABSMAX, bool PREFETCH, typename Release>
+// BIAS_IN_STAGE: bq_s points into `stage`, so a staged fp32 block must have been read by its TMA store before the
+// next block's bias values are exchanged there.
+template <int COLS, bool ABSMAX, bool PREFETCH, bool BIAS_IN_STAGE, typename Release>
 __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
                                               const CUtensorMap *tmap_yq, bool yq_tma, uint32_t taddr, int64_t row0,
                                               int64_t col0, const int32_t (&bqv)[COLS / 32], const float (&invv)[COLS / 32],
@@ -84,6 +86,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
         const int64_t nb = col0 + 32 * ci;
         const float inv = invv[ci];
         if (nb >= a.N || row0 >= a.M) return -1;  // warp-uniform: the block lies outside the matrix
+        if (BIAS_IN_STAGE && tma_store && lane == 0) tma_store_wait_read();
         // b_q of these 32 columns (one per lane, computed before the accumulator was ready) -> all lanes
         __syncwarp();
         bq_s[lane] = bqv[ci];
@@ -168,8 +171,8 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
         }
         if (a.Y == nullptr) return -1;
         if (tma_store) {
-            if (lane == 0) tma_store_wait_read();  // the previous block has left the staging buffer
-            __syncwarp();
+            if (!BIAS_IN_STAGE && lane == 0) tma_store_wait_read();  // the previous block has left the staging buffer
+            __syncwarp();  // (also: every lane has read the bias values before the block overwrites them)
             uint8_t *srow = stage + lane * 128;
 #pragma unroll
             for (int g = 0; g < 8; ++g)

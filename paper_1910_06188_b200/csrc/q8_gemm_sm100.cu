@@ -40,14 +40,17 @@ constexpr int kAccStages = 2;      // TMEM accumulator double buffering
 template <int BLOCK_N, int CTAS, int EW>
 struct Cfg {
     static constexpr int kEpilogueWarps = EW;
-    static constexpr int kThreads = 64 + 32 * EW;
+    static constexpr int kThreads = 96 + 32 * EW;  // two TMA producer warps, the MMA warp, EW epilogue warps
     static constexpr int kBRows = BLOCK_N / CTAS;  // W_q rows each CTA loads
     static constexpr int kABytes = BLOCK_M * BLOCK_K;
     static constexpr int kBBytes = kBRows * BLOCK_K;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStagingBytes = kEpilogueWarps * kStagingBytesPerWarp;
-    static constexpr int kBiasBytes = kEpilogueWarps * 32 * 4;  // b_q of the 32 columns a warp is working on
-    static constexpr int kRingBudget = 227 * 1024 - 1024 - 256 - kStagingBytes - kBiasBytes;  // left for the operand ring
+    // b_q of the 32 columns a warp is working on.  With 16 epilogue warps these 2 KB are what stands between four
+    // and five stages of the operand ring, so there the exchange happens inside the warp's own staging buffer.
+    static constexpr bool kBiasInStaging = EW == 16;
+    static constexpr int kBiasBytes = kBiasInStaging ? 0 : kEpilogueWarps * 32 * 4;
+    static constexpr int kRingBudget = 227 * 1024 - 1024 - 128 - kStagingBytes - kBiasBytes;  // left for the operand ring
     static constexpr int kStages = kRingBudget / kStageBytes > 8 ? 8 : kRingBudget / kStageBytes;
     static constexpr int kTmemCols = kAccStages * BLOCK_N < 32 ? 32 : kAccStages * BLOCK_N;
     static constexpr int kBarrierBytes = (2 * kStages + 2 * kAccStages) * 8 + 16;
@@ -67,7 +70,7 @@ struct Cfg {
 
 // ------------------------------------------------------------------ the kernel
 template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
-__global__ void __launch_bounds__(64 + 32 * EW, 1)
+__global__ void __launch_bounds__(96 + 32 * EW, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_w4,
                     const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_yq, GemmArgs a,
@@ -148,16 +151,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     grid_dependency_release_next(num_tiles <= 3 * num_units);  // up to three rounds of tiles count as small
     grid_dependency_wait();
 
-    if (warp == 0) {
-        // ---------------- TMA producer (each CTA loads its own rows) ----------------
-        // (a converged warp with one elected issuing lane, like the MMA warp below)
+    if (warp == 0 || warp == 2) {
+        // ---------------- TMA producers (each CTA loads its own rows) ----------------
+        // Two warps, each a converged warp with one elected issuing lane (like the MMA warp below): warp 0 takes the
+        // even k-blocks of the CTA's sequence of (tile, k-block) steps, warp 2 the odd ones.  One trip of a
+        // producer (wake up on the freed stage, arm the barrier, issue two tensor loads) takes 400 to 600 cycles,
+        // as long as the tensor cores need for the k-block (4 MMAs of 128 cycles), so a single producer cannot
+        // keep the ring full.
         {
+            const int p = warp >> 1;  // 0 or 1
             const uint32_t elected = elect_one();
-            int s = 0;
+            int s = p % C::kStages;
             uint32_t phase = 0;
             int issued = 0;
+            int64_t g = p;  // index of the step in the CTA's sequence (slot g % kStages, parity (g / kStages) & 1)
             bool ok = true;
-            for (int64_t tile = unit; ok && tile < num_tiles; tile += num_units) {
+            int kb = p;
+            int64_t tile = unit;
+            while (kb >= num_kb && tile < num_tiles) { kb -= num_kb; tile += num_units; }
+            while (ok && tile < num_tiles) {
                 int64_t m_idx, n_start;
                 int width;
                 decode(tile, m_idx, n_start, width);
@@ -166,7 +178,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 const int32_t n0 = (int32_t)(n_start + cta_rank * b_rows);
                 const CUtensorMap *map_w = width == BLOCK_N ? &tmap_w : (width * 2 == BLOCK_N ? &tmap_w2 : &tmap_w4);
                 const uint32_t stage_bytes = (uint32_t)(C::kABytes + b_rows * BLOCK_K);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (; kb < num_kb; kb += 2) {
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(empty_bar + s), phase ^ 1u, abort_flag, a.status));
                     if (!ok) break;
                     const uint32_t fb = smem_u32(full_bar + s);
@@ -183,16 +195,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                         tma_load_2d_pair_elected(elected, dst_b, map_w, kb * BLOCK_K, n0, fb_leader);
                     }
                     ++issued;
-                    if (++s == C::kStages) { s = 0; phase ^= 1u; }
+                    g += 2;
+                    s += 2;
+                    if (s >= C::kStages) { s -= C::kStages; phase ^= 1u; }
                 }
+                if (!ok) break;
+                do { kb -= num_kb; tile += num_units; } while (kb >= num_kb && tile < num_tiles);
             }
             if (!ok) {
-                // Aborting: let the copies already issued land before the CTA gives up its shared memory.
+                // Aborting: let this warp's copies already issued land before the CTA gives up its shared memory.
                 const uint64_t t0 = global_timer_ns();
                 if (CTAS == 1 || leader) {
-                    const int pending = issued < C::kStages ? issued : C::kStages;
+                    const int mine = (C::kStages + 1) / 2;  // at most this many of a producer's steps are in flight
+                    const int pending = issued < mine ? issued : mine;
                     for (int i = 0; i < pending; ++i) {
-                        const int k = issued - 1 - i;  // the i-th most recent k-block
+                        const int64_t k = g - 2 * (i + 1);  // the i-th most recent step of this producer
                         const uint32_t par = (uint32_t)((k / C::kStages) & 1);
                         while (!mbar_try_wait(smem_u32(full_bar + k % C::kStages), par) &&
                                global_timer_ns() - t0 < 50000000ull) {}
@@ -261,7 +278,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         }
     } else {
         // ---------------- epilogue ----------------
-        const int ew = warp - 2;       // 0 .. EW-1
+        const int ew = warp - 3;       // 0 .. EW-1
         const int quarter = warp & 3;  // TMEM lanes this warp may touch: 32*quarter .. +31
         const int col_group = ew >> 2;  // which share of the tile's columns this warp takes
         const float S_x = __ldg(a.S_x);
@@ -272,7 +289,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             return __fmul_rn(S_x, __ldg(a.S_w + seg));
         };
         uint8_t *stage = smem_stage + ew * kStagingBytesPerWarp;
-        int32_t *bq_s = smem_bq + ew * 32;
+        // (inside the staging buffer: the first 128 bytes when fp32 blocks are staged, which are free once the
+        // previous block's TMA store has read them, or past the 32 x 64 staged Int8 bytes of an Int8-only tile)
+        int32_t *bq_s = C::kBiasInStaging ? reinterpret_cast<int32_t *>(stage + (a.Y == nullptr ? 2048 : 0)) : smem_bq + ew * 32;
         int as = 0;
         uint32_t aphase = 0;
         bool ok = true;
@@ -338,7 +357,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     a, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                     m0 + quarter * 32, n0 + col_off, bqv, invv, bq_s, lane, cpw / 32, release, absmax_run);
             else if (active)
-                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8)>(a, &tmap_y, tma_store == 1, &tmap_yq, yq_tma != 0,
+                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8), C::kBiasInStaging>(a, &tmap_y, tma_store == 1, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                                                m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release,
                                                absmax_run);
@@ -368,7 +387,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 // ------------------------------------------------------------------ host side
 int g_force_block_n = 0, g_force_ctas = 0;  // set by q8_tune_gemm_tile(); 0 = choose automatically
 int g_force_epilogue_warps = 0;            // 0 automatic, else 8 or 16 (cta_group::2 kernel only)
-bool g_direct_store = false;               // fp32-only output stored from the 16x256b fragment layout, no staging
+int g_direct_store = -1;                   // fp32-only output stored straight from registers: 1 yes, 0 no, -1 automatic
 bool g_tail_split_enabled = true;          // cut the tiles of a partial last round into narrower ones
 
 template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
@@ -442,7 +461,11 @@ cudaError_t launch_cfg_impl(const GemmArgs &a, cudaStream_t s)
     }
     // the TMA store needs a 16-byte aligned base and row pitch; otherwise lanes store their rows directly
     int tma_store = a.Y != nullptr && ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
-    if (g_direct_store && a.Y != nullptr && a.Yq == nullptr && ((a.N & 1) == 0) &&
+    // Automatic choice: with a long main loop (the 8-warp epilogue of the CTA pair, K > 2048) the unstaged stores
+    // are a little faster (FFN2 75.1 -> 73.7 us: no staging traffic in shared memory, which the operand ring and
+    // the tensor cores already load fully); with a short one the staged TMA stores win (QKV 79.5 against 85.7 us).
+    const bool direct = g_direct_store < 0 ? (CTAS == 2 && EW == 8) : g_direct_store != 0;
+    if (direct && a.Y != nullptr && a.Yq == nullptr && ((a.N & 1) == 0) &&
         ((reinterpret_cast<uintptr_t>(a.Y) & 7u) == 0)) {
         tma_store = 2;
         ty = tx;
@@ -517,7 +540,7 @@ void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps)
 }
 
 void set_gemm_tail_split(bool enable) { g_tail_split_enabled = enable; }
-void set_gemm_direct_store(bool enable) { g_direct_store = enable; }
+void set_gemm_direct_store(int mode) { g_direct_store = mode < 0 ? -1 : (mode != 0); }
 void set_gemm_epilogue_warps(int warps) { g_force_epilogue_warps = warps; }
 
 bool tcgen05_gemm_supported(const GemmArgs &a)

@@ -101,7 +101,7 @@ int32_t *attention_status_word();  // device word that receives Q8_ERR_TIMEOUT f
 bool tcgen05_gemm_supported(const GemmArgs &a);
 void set_gemm_tile_override(int block_n, int ctas, int epilogue_warps = 0);  // 0, 0 = automatic choice
 void set_gemm_tail_split(bool enable);
-void set_gemm_direct_store(bool enable);
+void set_gemm_direct_store(int mode);
 void set_gemm_epilogue_warps(int warps);  // 0 automatic, 8 or 16
 cudaError_t launch_gemm_tcgen05(const GemmArgs &a, cudaStream_t s);  // q8_gemm_sm100.cu
 cudaError_t launch_gemm_generic(const GemmArgs &a, cudaStream_t s);  // q8_gemm_generic.cu

@@ -279,3 +279,36 @@ def test_empty_problem_is_a_noop():
     assert xq.numel() == 0
     out = q8.q8_embedding(torch.empty(0, dtype=torch.int32, device="cuda"), Wq, S)
     assert out.shape == (0, 16)
+
+
+@pytest.mark.parametrize("direct", [False, True])
+@pytest.mark.parametrize("warps", [8, 16])
+def test_both_output_store_paths_of_the_pair_kernel_match_the_oracle(direct, warps):
+    """fp32 output staged in shared memory and TMA-stored, or stored straight from the 16 x 256 bit accumulator
+    fragments: same values (ragged M, N, K; odd tails; with and without GELU), also in the debug accumulator."""
+    from tests.gpu_util import check_linear
+    try:
+        q8.q8_tune_gemm_tile(256, 2)
+        q8.q8_tune_gemm_epilogue_warps(warps)
+        q8.q8_tune_gemm_direct_store(direct)
+        for (Mm, Nn, Kk, act) in [(700, 520, 272, 1), (515, 1030, 144, 0), (300, 130, 256, 0), (129, 34, 64, 1)]:
+            X = synth.activation(Mm, Kk, seed=1400 + Mm)
+            W = synth.weight(Nn, Kk, seed=1401 + Mm)
+            bb = synth.bias(Nn, seed=1402 + Mm)
+            info = check_linear(X, W, bb, act=act)
+            assert (info["block_n"], info["ctas"]) == (256, 2)
+    finally:
+        q8.q8_tune_gemm_direct_store(None)
+        q8.q8_tune_gemm_epilogue_warps(0)
+        q8.q8_tune_gemm_tile(0, 0)
+
+
+def test_l2_operand_probe_runs_and_rejects_bad_arguments():
+    buf = torch.zeros((1024, 1024), dtype=torch.int8, device="cuda")
+    r = q8.q8_measure_l2_operand_peak(buf, 1024, 1024, boxes_per_sm=256, sms_used=4, producers=2)
+    assert r["gbs"] > 0 and r["elapsed_ms"] > 0
+    for bad in [dict(rows=100), dict(K=100), dict(producers=5), dict(sms_used=100000)]:
+        kw = dict(rows=1024, K=1024, boxes_per_sm=16, sms_used=1, producers=1)
+        kw.update(bad)
+        with pytest.raises(q8.Q8Error):
+            q8.q8_measure_l2_operand_peak(buf, **kw)
