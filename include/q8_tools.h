@@ -33,7 +33,8 @@ void q8_tune_gemm_tail_split(int enable);
 
 /* Tuning / test hook for the way the tcgen05 GEMM writes a plain fp32 output (no Int8 copy asked for).
  * mode 1: each epilogue warp reads its accumulator block in the 16 x 256 bit fragment layout and stores it
- * straight from registers, every 32-byte sector written whole by four neighbouring lanes; mode 0: the block
+ * straight from registers, every 32-byte sector written whole by four neighbouring lanes (CTA-pair kernel only, and
+ * only when neither an Int8 copy nor the debug accumulator is asked for); mode 0: the block
  * is staged in shared memory and leaves as a TMA store; mode < 0 (the default): automatic, unstaged only for the
  * CTA-pair kernel with the 8-warp epilogue (K > 2048), where it measured 2 % faster.  Results do not depend on
  * it.  Not thread-safe. */
@@ -42,6 +43,11 @@ void q8_tune_gemm_direct_store(int mode);
 /* Into how many narrower tiles each tile of the last round was cut by the most recent tcgen05 GEMM launch
  * of this host thread: 1 (not cut), 2 or 4. */
 int q8_last_launch_tail_split(void);
+
+/* How the most recent tcgen05 GEMM launch of this host thread wrote its fp32 output: 0 every lane stored its own
+ * row (Y not aligned for a TMA store, or no fp32 output), 1 staged in shared memory and stored by TMA, 2 stored
+ * straight from the accumulator fragments (see q8_tune_gemm_direct_store). */
+int q8_last_launch_store_mode(void);
 
 /* Tuning / test hook: q8_attention / q8_attention_quant use the tensor-core kernel when the shape allows it
  * (non-zero, the default) or always the CUDA-core fp32 kernel (0), for later calls in this process. */

@@ -59,6 +59,7 @@ SIGNATURES = {
     "q8_attention_status_word": (_int, [C.POINTER(C.c_void_p)]),
     "q8_tune_gemm_epilogue_warps": (_int, [_int]),
     "q8_last_launch_tail_split": (_int, []),
+    "q8_last_launch_store_mode": (_int, []),
     "q8_measure_hbm_peak": (_int, [C.c_void_p, C.c_size_t, _int, _int, C.POINTER(C.c_double), C.POINTER(C.c_double),
                                    C.c_void_p]),
     "q8_measure_l2_operand_peak": (_int, [C.c_void_p, C.c_int64, C.c_int64, _int, _int, _int, C.POINTER(C.c_double),
@@ -566,6 +567,11 @@ def q8_tune_gemm_tail_split(enable: bool = True) -> None:
 def q8_tune_gemm_direct_store(mode: Optional[bool] = None) -> None:
     """fp32-only GEMM output stored straight from registers (True), staged and TMA-stored (False) or automatic (None)."""
     load().q8_tune_gemm_direct_store(-1 if mode is None else (1 if mode else 0))
+
+
+def q8_last_launch_store_mode() -> int:
+    """0 lanes stored their rows, 1 staged + TMA store, 2 stored straight from the accumulator fragments."""
+    return int(load().q8_last_launch_store_mode())
 
 
 def q8_last_launch_tail_split() -> int:

@@ -510,5 +510,6 @@ void q8_tune_gemm_tail_split(int enable) { set_gemm_tail_split(enable != 0); }
 void q8_tune_gemm_direct_store(int mode) { set_gemm_direct_store(mode); }
 
 int q8_last_launch_tail_split(void) { return last_launch_info().tail_split; }
+int q8_last_launch_store_mode(void) { return last_launch_info().store_mode; }
 
 }  // extern "C"

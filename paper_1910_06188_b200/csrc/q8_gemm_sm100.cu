@@ -69,7 +69,13 @@ struct Cfg {
 };
 
 // ------------------------------------------------------------------ the kernel
-template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
+// OUT: what the epilogue writes.  kOutPlain: fp32 Y, staged in shared memory and stored by TMA (or by the lanes
+// when Y is not aligned for that); kOutFull: the same plus the Int8 copy and the debug copy of the accumulator, as
+// asked for; kOutDirect: fp32 Y stored straight from the accumulator fragments.  Separate instantiations, so that
+// the plain layer does not carry the registers of the paths it does not take.
+constexpr int kOutPlain = 0, kOutFull = 1, kOutDirect = 2;
+
+template <int BLOCK_N, int CTAS, int EW, bool ABSMAX, int OUT>
 __global__ void __launch_bounds__(96 + 32 * EW, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_w4,
@@ -352,12 +358,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     else mbar_arrive(smem_u32(tmem_empty_bar + as));
                 }
             };
-            if (active && tma_store == 2)
+            if (active && OUT == kOutDirect)
                 epilogue_warp_direct<C::kColsPerWarp, ABSMAX>(
                     a, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                     m0 + quarter * 32, n0 + col_off, bqv, invv, bq_s, lane, cpw / 32, release, absmax_run);
             else if (active)
-                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8), C::kBiasInStaging>(a, &tmap_y, tma_store == 1, &tmap_yq, yq_tma != 0,
+                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8), C::kBiasInStaging, OUT == kOutPlain>(a, &tmap_y, tma_store == 1, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                                                m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release,
                                                absmax_run);
@@ -390,23 +396,45 @@ int g_force_epilogue_warps = 0;            // 0 automatic, else 8 or 16 (cta_gro
 int g_direct_store = -1;                   // fp32-only output stored straight from registers: 1 yes, 0 no, -1 automatic
 bool g_tail_split_enabled = true;          // cut the tiles of a partial last round into narrower ones
 
-template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
+template <int BLOCK_N, int CTAS, int EW, bool ABSMAX, int OUT>
 cudaError_t launch_cfg_impl(const GemmArgs &a, cudaStream_t s);
 
-// The layer that also reports max|y| (Sec. 4.1 chained dynamically) runs its own instantiation of the kernel.
+// Unstaged stores of a plain fp32 output: chosen automatically where they measured faster, i.e. with a long main loop
+// (the 8-warp epilogue of the CTA pair, K > 2048: FFN2 75.1 -> 73.7 us, no staging traffic in shared memory, which the
+// operand ring and the tensor cores already load fully); with a short one the staged TMA stores win (QKV 79.5
+// against 85.7 us).  The pair kernels alone have the instantiation.
+template <int CTAS, int EW>
+bool wants_direct_store(const GemmArgs &a)
+{
+    const bool direct = g_direct_store < 0 ? (CTAS == 2 && EW == 8) : g_direct_store != 0;
+    return CTAS == 2 && direct && a.Y != nullptr && a.Yq == nullptr && a.dbg_acc == nullptr && ((a.N & 1) == 0) &&
+           ((reinterpret_cast<uintptr_t>(a.Y) & 7u) == 0);
+}
+
+// The layer that also reports max|y| (Sec. 4.1 chained dynamically) and each output mode run their own
+// instantiation of the kernel.
+template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
+cudaError_t launch_cfg_out(const GemmArgs &a, cudaStream_t s)
+{
+    if (a.Yq != nullptr || a.dbg_acc != nullptr) return launch_cfg_impl<BLOCK_N, CTAS, EW, ABSMAX, kOutFull>(a, s);
+    if constexpr (CTAS == 2) {
+        if (wants_direct_store<CTAS, EW>(a)) return launch_cfg_impl<BLOCK_N, CTAS, EW, ABSMAX, kOutDirect>(a, s);
+    }
+    return launch_cfg_impl<BLOCK_N, CTAS, EW, ABSMAX, kOutPlain>(a, s);
+}
 template <int BLOCK_N, int CTAS, int EW = 8>
 cudaError_t launch_cfg(const GemmArgs &a, cudaStream_t s)
 {
-    return a.y_absmax != nullptr ? launch_cfg_impl<BLOCK_N, CTAS, EW, true>(a, s)
-                                 : launch_cfg_impl<BLOCK_N, CTAS, EW, false>(a, s);
+    return a.y_absmax != nullptr ? launch_cfg_out<BLOCK_N, CTAS, EW, true>(a, s)
+                                 : launch_cfg_out<BLOCK_N, CTAS, EW, false>(a, s);
 }
 
-template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
+template <int BLOCK_N, int CTAS, int EW, bool ABSMAX, int OUT>
 cudaError_t launch_cfg_impl(const GemmArgs &a, cudaStream_t s)
 {
     using C = Cfg<BLOCK_N, CTAS, EW>;
     constexpr int kThreads = C::kThreads;
-    auto kernel = gemm_tcgen05_kernel<BLOCK_N, CTAS, EW, ABSMAX>;
+    auto kernel = gemm_tcgen05_kernel<BLOCK_N, CTAS, EW, ABSMAX, OUT>;
     static bool attr_set[64] = {};  // the opt-in shared-memory size is a per-device, per-function attribute
     static int max_units[64] = {};  // co-resident CTAs (CTAS = 1) or CTA pairs (CTAS = 2) on the device
     int dev = 0;
@@ -460,16 +488,9 @@ cudaError_t launch_cfg_impl(const GemmArgs &a, cudaStream_t s)
         tw4 = tw;
     }
     // the TMA store needs a 16-byte aligned base and row pitch; otherwise lanes store their rows directly
-    int tma_store = a.Y != nullptr && ((a.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
-    // Automatic choice: with a long main loop (the 8-warp epilogue of the CTA pair, K > 2048) the unstaged stores
-    // are a little faster (FFN2 75.1 -> 73.7 us: no staging traffic in shared memory, which the operand ring and
-    // the tensor cores already load fully); with a short one the staged TMA stores win (QKV 79.5 against 85.7 us).
-    const bool direct = g_direct_store < 0 ? (CTAS == 2 && EW == 8) : g_direct_store != 0;
-    if (direct && a.Y != nullptr && a.Yq == nullptr && ((a.N & 1) == 0) &&
-        ((reinterpret_cast<uintptr_t>(a.Y) & 7u) == 0)) {
-        tma_store = 2;
-        ty = tx;
-    } else if (tma_store) {
+    int tma_store = OUT != kOutDirect && a.Y != nullptr && ((a.N & 3) == 0) &&
+                    ((reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0);
+    if (tma_store) {
         if (!make_tmap_out(&ty, a.Y, a.M, a.N)) return cudaErrorInvalidValue;
     } else {
         ty = tx;  // never dereferenced
@@ -503,6 +524,7 @@ cudaError_t launch_cfg_impl(const GemmArgs &a, cudaStream_t s)
     li.epilogue_warps = EW;
     li.grid = units * CTAS;
     li.tail_split = split;
+    li.store_mode = OUT == kOutDirect ? 2 : tma_store;
     li.launches += 1;
     return e;
 }

@@ -53,6 +53,7 @@ struct LaunchInfo {
     int epilogue_warps = 0;
     int grid = 0;
     int tail_split = 1;  // tiles of the last scheduling round cut into this many narrower ones
+    int store_mode = 0;  // fp32 output of the tcgen05 GEMM: 0 stored by the lanes, 1 staged + TMA store, 2 unstaged
 };
 LaunchInfo &last_launch_info();
 

@@ -285,8 +285,9 @@ def test_empty_problem_is_a_noop():
 @pytest.mark.parametrize("warps", [8, 16])
 def test_both_output_store_paths_of_the_pair_kernel_match_the_oracle(direct, warps):
     """fp32 output staged in shared memory and TMA-stored, or stored straight from the 16 x 256 bit accumulator
-    fragments: same values (ragged M, N, K; odd tails; with and without GELU), also in the debug accumulator."""
-    from tests.gpu_util import check_linear
+    fragments: the oracle's values either way (ragged M, N, K; odd tails; with and without GELU).  A call that also
+    wants the debug accumulator takes the staged path whatever the hook says."""
+    from tests.gpu_util import check_linear, assert_close_fp, dev
     try:
         q8.q8_tune_gemm_tile(256, 2)
         q8.q8_tune_gemm_epilogue_warps(warps)
@@ -295,8 +296,20 @@ def test_both_output_store_paths_of_the_pair_kernel_match_the_oracle(direct, war
             X = synth.activation(Mm, Kk, seed=1400 + Mm)
             W = synth.weight(Nn, Kk, seed=1401 + Mm)
             bb = synth.bias(Nn, seed=1402 + Mm)
-            info = check_linear(X, W, bb, act=act)
+            info = check_linear(X, W, bb, act=act)  # with dbg_Xq / dbg_acc
             assert (info["block_n"], info["ctas"]) == (256, 2)
+            staged = 1 if Nn % 4 == 0 else 0  # a TMA store needs a 16-byte row pitch
+            assert q8.q8_last_launch_store_mode() == staged
+            # the plain call: Y only
+            Wq_ref, S_w_ref, _ = o.quantize_weight(W)
+            ref = o.linear(X, Wq_ref, S_w_ref, None, bb, act)
+            Wq, S_w = q8.q8_quantize_weight(dev(W))
+            Ybuf = torch.full((Mm * Nn + 64,), 12345.0, dtype=torch.float32, device="cuda")
+            Y = Ybuf[: Mm * Nn].view(Mm, Nn)
+            q8.q8_linear(dev(X), Wq, S_w, None, dev(bb), act, Y=Y)
+            assert q8.q8_last_launch_store_mode() == (2 if direct else staged)
+            assert_close_fp(Y.cpu().numpy(), ref["y"], "Y")
+            assert torch.all(Ybuf[Mm * Nn:] == 12345.0)  # nothing stored past the matrix
     finally:
         q8.q8_tune_gemm_direct_store(None)
         q8.q8_tune_gemm_epilogue_warps(0)
