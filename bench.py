@@ -40,7 +40,7 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of the tcgen05 GEMM per launch on the BERT-Large FC set, from the
 # ncu captures summarised in profiles/gemm_tcgen05_dram_traffic_m24576.md (one layer resident per capture).  Below the
 # algorithmic bytes because part of each output is still dirty in the 126 MB L2 when the kernel ends.
-GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 269975040, "attn_out": 67070464, "ffn1": 372139008, "ffn2": 162752768}}
+GEMM_DRAM_TRAFFIC = {"bert_large_fc": {"qkv": 269605632, "attn_out": 66903040, "ffn1": 371766784, "ffn2": 164554496}}
 NOMINAL_INT8_OVER_BF16 = 2.0  # dense tensor peak ratio int8 : bf16 (4.5 : 2.25 POPS nominal)
 GEMM_REPS = 4   # launches per event pair in the per-kernel pass
 QUANT_REPS = 4  # times each group of equal-sized quantise passes is repeated per event pair
@@ -575,6 +575,7 @@ def run_ours(args):
     # the sustained one when the clock sagged under the power cap.
     at_max_clock = bool(clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] >= 0.97 * clocks["sm_max_mhz"])
     peak_key = "bf16_tflops" if at_max_clock else "bf16_tflops_sustained"
+    sm_hz = float(clocks.get("sm_mhz") or 1965.0) * 1e6  # SM clock sampled while the timed region ran
     int8_peak = float(peaks.get(peak_key, FALLBACK_PEAKS[peak_key])) * NOMINAL_INT8_OVER_BF16
     int8_peak_sustained = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"])) * NOMINAL_INT8_OVER_BF16
     hbm_peak = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
@@ -598,9 +599,6 @@ def run_ours(args):
     for L in layers:
         tiles_m, tiles_n = -(-L["M"] // 256), -(-L["N"] // 256)
         fabric_bytes.append(tiles_m * tiles_n * 512 * L["K"] + 4 * L["M"] * L["N"])
-    # Bytes that pass through the L2 data arrays per launch: the operand loads above, and the fp32 output twice
-    # (written into L2 by the SMs, read out of it again on its way to HBM).
-    l2_bytes = [fb + 4 * L["M"] * L["N"] for L, fb in zip(layers, fabric_bytes)]
     # Issue-bound Int8 rate of the tensor cores on this device (operands resident in shared memory), measured now
     mma_peak = None
     if world == 1:
@@ -641,6 +639,18 @@ def run_ours(args):
             "what": "store-only and load-only rates of a grid-stride 16-byte kernel over 1 GiB (q8_measure_hbm_peak); per "
                     "layer floor = max(2MNK / Int8 peak, 4MN / store-only rate)",
         }
+    # What L2 can feed the SMs through TMA, measured now on an L2-resident matrix of the first layer's operand shape
+    l2_probe = None
+    n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    if world == 1:
+        pm = torch.zeros((4096, 1024), dtype=torch.int8, device=dev)
+        r4 = q8.q8_measure_l2_operand_peak(pm, 4096, 1024, boxes_per_sm=2048, producers=4)
+        r1 = q8.q8_measure_l2_operand_peak(pm, 4096, 1024, boxes_per_sm=2048, producers=1)
+        del pm
+        l2_probe = {"tbs_all_sms_4_issuing_warps": r4["gbs"] / 1e3, "gbs_per_sm_4_issuing_warps": r4["gbs"] / n_sms,
+                    "gbs_per_sm_1_issuing_warp": r1["gbs"] / n_sms,
+                    "needed_gbs_per_sm_at_full_int8_rate": 64.0 * sm_hz / 1e9,
+                    "what": "q8_measure_l2_operand_peak: 128-row x 128-byte boxes, 12 stages in flight per SM"}
     emb_ms = t_emb / ksteps
     emb_cold_ms = t_emb_cold / ksteps
     emb_bytes = 5.0 * M * H + 4.0 * M
@@ -674,17 +684,23 @@ def run_ours(args):
             "bytes_per_launch_mean": sum(fabric_bytes) / len(fabric_bytes),
             "achieved_tbs": sum(fabric_bytes) / (sum(gemm_ms) * 1e-3) / 1e12,
             "by_layer_tbs": {L["name"]: fb / (gm * 1e-3) / 1e12 for L, fb, gm in zip(layers, fabric_bytes, gemm_ms)},
-            "note": "operand re-loads of the 256 x 256 pair tiles plus the fp32 output, all through L2; with the epilogue "
-                    "left out the main loop alone moves operands at 12.6-12.9 TB/s (graph-replayed launches)",
+            "l2_operand_probe": l2_probe,
+            "note": "operand re-loads of the 256 x 256 pair tiles plus the fp32 output, all through L2.  L2 itself is not the "
+                    "limit: the probe (TMA loads of the GEMM's operand boxes by every SM, nothing else running, measured "
+                    "now) delivers well above the 64 B/clk/SM the main loop asks for at the full Int8 rate",
         },
-        "l2_throughput": {
-            "bytes_per_launch_mean": sum(l2_bytes) / len(l2_bytes),
-            "achieved_tbs": sum(l2_bytes) / (sum(gemm_ms) * 1e-3) / 1e12,
-            "by_layer_tbs": {L["name"]: lb / (gm * 1e-3) / 1e12 for L, lb, gm in zip(layers, l2_bytes, gemm_ms)},
-            "reference_tbs": 12.9,
-            "note": "operand loads (M N K / 128 bytes with 256 x 256 pair tiles) + 2 x the fp32 output (into L2, and out of it "
-                    "to HBM); the main loop alone, without any epilogue, reads operands from L2 at 12.6-12.9 TB/s on this "
-                    "part, and every full-size shape lands within 10 % of (loads + 2 Y) / 12.9 TB/s",
+        "sm_side_limits": {
+            "write_port_bytes_per_clk_per_sm": 32,
+            "y_store_us_at_write_port": {L["name"]: 4.0 * L["M"] * L["N"] / (n_sms * 32.0 * sm_hz) * 1e6 for L in layers},
+            "main_loop_only_us": {"qkv": 44.6, "attn_out": 18.7, "ffn1": 58.3, "ffn2": 66.4} if args.workload == "bert_large_fc" else None,
+            "note": "an SM writes to L2 at no more than 32 bytes per clock (ncu: l1tex__m_l1tex2xbar_write_bytes peak), "
+                    "whether by TMA store or by st.global, so the fp32 output of a layer occupies that port for "
+                    "y_store_us_at_write_port (at the SM clock sampled in this run); measured kernel times are close to "
+                    "main_loop_only_us (the same kernel with the epilogue reduced to handing the accumulator back, a work "
+                    "copy, graph-replayed) plus that port time, i.e. the two do not overlap.  The main loop alone runs at "
+                    "about three quarters of the issue-bound Int8 rate: TMA writes 64 B/clk/SM into shared memory while "
+                    "the tensor cores read 64 B/clk/SM from it (with no loads the same loop takes 54.5 us on FFN2, with "
+                    "only the B tiles 56.3, with both operands 66.4)",
         },
         "note": "GEMM times: CUDA events around a graph replay of %d back-to-back launches of the layer (X_q just written by the quantise "
                 "pass, output streamed to HBM); quantise times: events around the back-to-back group of equal-sized layers "

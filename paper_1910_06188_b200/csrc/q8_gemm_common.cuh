@@ -59,10 +59,13 @@ __device__ __forceinline__ void gelu_fast_x2(uint64_t y2, float &out_lo, float &
 // warp walks four blocks per tile; with two blocks per warp it measured 1 % slower).
 // BIAS_IN_STAGE: bq_s points into `stage`, so a staged fp32 block must have been read by its TMA store before the
 // next block's bias values are exchanged there.
-// LEAN: the plain layer (fp32 Y only): the Int8 copy and the debug copy of the accumulator are compiled out, which
-// keeps the 16-warp kernel (96 registers per thread) free of spills; a spilled value is reloaded from local memory
-// in every block, and under the main loop's traffic that load is not a cache hit.
-template <int COLS, bool ABSMAX, bool PREFETCH, bool BIAS_IN_STAGE, bool LEAN, typename Release>
+// OUT: which outputs the instantiation can write.  kOutPlain: the fp32 Y only; kOutInt8: the Int8 copy only (the
+// fused FFN1 of a forward whose next layer is quantised); kOutFull: whatever the call asks for (fp32, Int8, the
+// debug copy of the accumulator).  Compiling the other paths out keeps the 16-warp kernel (96 registers per thread)
+// free of spills; a spilled value is reloaded from local memory in every block, and under the main loop's traffic
+// that load is not a cache hit.
+constexpr int kOutPlain = 0, kOutFull = 1, kOutDirect = 2, kOutInt8 = 3;
+template <int COLS, bool ABSMAX, bool PREFETCH, bool BIAS_IN_STAGE, int OUT, typename Release>
 __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorMap *tmap_y, bool tma_store,
                                               const CUtensorMap *tmap_yq, bool yq_tma, uint32_t taddr, int64_t row0,
                                               int64_t col0, const int32_t (&bqv)[COLS / 32], const float (&invv)[COLS / 32],
@@ -72,13 +75,14 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
     constexpr int NCHUNK = COLS / 32;  // compile-time maximum; this tile has nch <= NCHUNK blocks (warp-uniform)
     const int64_t row = row0 + lane;
     const bool row_ok = row < a.M;
-    const float S_y = (!LEAN && a.Yq != nullptr) ? __ldg(a.S_y) : 1.0f;
+    constexpr bool kHasY = OUT != kOutInt8, kHasYq = OUT == kOutFull || OUT == kOutInt8, kHasDbg = OUT == kOutFull;
+    const float S_y = (kHasYq && a.Yq != nullptr) ? __ldg(a.S_y) : 1.0f;
     const bool yq_vec = ((a.N & 15) == 0) && ((reinterpret_cast<uintptr_t>(a.Yq) & 15u) == 0);
     // Int8-only output of a full-width tile: the warp's 32 x COLS bytes are collected in its staging buffer (free,
     // since no fp32 block is staged) in the swizzled layout of the Int8 output tensor map and leave as one TMA
     // store of whole 64- or 128-byte row pieces instead of 32 separate 16-byte stores per lane and block.
     constexpr bool kYqStageable = COLS == 64 || COLS == 128;
-    const bool yq_staged = !LEAN && kYqStageable && yq_tma && nch == NCHUNK;
+    const bool yq_staged = kHasYq && kYqStageable && yq_tma && nch == NCHUNK;
     const int yq_xor = COLS == 128 ? (lane & 7) : ((lane >> 1) & 3);  // 128-byte / 64-byte swizzle of row `lane`
     bool yq_pending = false;
 
@@ -102,7 +106,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
             v[4 * g + 2] = (uint32_t)add_wrap((int32_t)v[4 * g + 2], b.z);
             v[4 * g + 3] = (uint32_t)add_wrap((int32_t)v[4 * g + 3], b.w);
         }
-        if (!LEAN && a.dbg_acc != nullptr && row_ok) {
+        if (kHasDbg && a.dbg_acc != nullptr && row_ok) {
             int32_t *drow = a.dbg_acc + row * a.N + nb;
 #pragma unroll
             for (int j = 0; j < 32; ++j)
@@ -130,7 +134,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
             for (int j = 0; j < 32; ++j)
                 if (whole || nb + j < a.N) absmax_run = fmaxf(absmax_run, fabsf(__uint_as_float(v[j])));
         }
-        if (!LEAN && a.Yq != nullptr && row_ok) {
+        if (kHasYq && a.Yq != nullptr && row_ok) {
             // re-quantised output for the next quantised layer: Eq. 1 at that layer's activation scale
             int8_t *qrow = a.Yq + row * a.N + nb;
             if (yq_staged) {
@@ -154,7 +158,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
                     if (nb + j < a.N) qrow[j] = (int8_t)quantize_value(__uint_as_float(v[j]), S_y);
             }
         }
-        if (!LEAN && yq_staged) {
+        if (kHasYq && yq_staged) {
             if (!yq_pending) {
                 if (lane == 0) tma_store_wait_read();  // the previous tile has left the staging buffer
                 __syncwarp();
@@ -172,7 +176,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
                 quantize_pack4(__uint_as_float(v[24]), __uint_as_float(v[25]), __uint_as_float(v[26]), __uint_as_float(v[27]), S_y),
                 quantize_pack4(__uint_as_float(v[28]), __uint_as_float(v[29]), __uint_as_float(v[30]), __uint_as_float(v[31]), S_y));
         }
-        if (a.Y == nullptr) return -1;
+        if (!kHasY || a.Y == nullptr) return -1;
         if (tma_store) {
             if (!BIAS_IN_STAGE && lane == 0) tma_store_wait_read();  // the previous block has left the staging buffer
             __syncwarp();  // (also: every lane has read the bias values before the block overwrites them)
@@ -211,7 +215,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
         if (PREFETCH && ci + 1 < nch) tmem_ld_32x32(taddr + (uint32_t)(32 * (ci + 1)), v);
         if (staged_at >= 0) issue_store(staged_at);
     }
-    if (!LEAN && yq_pending) {
+    if (kHasYq && yq_pending) {
         // blocks beyond column N were never staged; the store clips them (and rows past M) at the matrix edge
         fence_proxy_async_smem();
         __syncwarp();
@@ -222,7 +226,7 @@ __device__ __forceinline__ void epilogue_warp(const GemmArgs &a, const CUtensorM
 // The same work for the plain fp32 output (no Int8 copy), without the shared-memory staging: the accumulator block is
 // read in the 16x256b fragment layout, where four neighbouring lanes hold 32 contiguous bytes of a row, so each lane
 // stores its pairs straight to Y (8-byte stores, every sector written whole by one instruction).  No proxy fence,
-// no TMA store, no staging buffer to wait for.  Needs an even N and an 8-byte aligned Y; like the LEAN form of the
+// no TMA store, no staging buffer to wait for.  Needs an even N and an 8-byte aligned Y; like the plain form of the
 // staged epilogue it writes Y only (a call that wants the Int8 or the debug copy takes the staged path).
 template <int COLS, bool ABSMAX, typename Release>
 __device__ __forceinline__ void epilogue_warp_direct(const GemmArgs &a, uint32_t taddr, int64_t row0, int64_t col0,

@@ -70,10 +70,9 @@ struct Cfg {
 
 // ------------------------------------------------------------------ the kernel
 // OUT: what the epilogue writes.  kOutPlain: fp32 Y, staged in shared memory and stored by TMA (or by the lanes
-// when Y is not aligned for that); kOutFull: the same plus the Int8 copy and the debug copy of the accumulator, as
-// asked for; kOutDirect: fp32 Y stored straight from the accumulator fragments.  Separate instantiations, so that
-// the plain layer does not carry the registers of the paths it does not take.
-constexpr int kOutPlain = 0, kOutFull = 1, kOutDirect = 2;
+// when Y is not aligned for that); kOutInt8: only the Int8 copy; kOutFull: fp32 and / or Int8 and / or the debug copy
+// of the accumulator, as asked for; kOutDirect: fp32 Y stored straight from the accumulator fragments.  Separate
+// instantiations, so that a layer does not carry the registers of the paths it does not take.
 
 template <int BLOCK_N, int CTAS, int EW, bool ABSMAX, int OUT>
 __global__ void __launch_bounds__(96 + 32 * EW, 1)
@@ -363,7 +362,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     a, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                     m0 + quarter * 32, n0 + col_off, bqv, invv, bq_s, lane, cpw / 32, release, absmax_run);
             else if (active)
-                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8), C::kBiasInStaging, OUT == kOutPlain>(a, &tmap_y, tma_store == 1, &tmap_yq, yq_tma != 0,
+                epilogue_warp<C::kColsPerWarp, ABSMAX, (EW == 8), C::kBiasInStaging, OUT>(a, &tmap_y, tma_store == 1, &tmap_yq, yq_tma != 0,
                                                tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(as * BLOCK_N + col_off),
                                                m0 + quarter * 32, n0 + col_off, bqv, invv, stage, bq_s, lane, cpw / 32, release,
                                                absmax_run);
@@ -416,6 +415,8 @@ bool wants_direct_store(const GemmArgs &a)
 template <int BLOCK_N, int CTAS, int EW, bool ABSMAX>
 cudaError_t launch_cfg_out(const GemmArgs &a, cudaStream_t s)
 {
+    if (a.Yq != nullptr && a.Y == nullptr && a.dbg_acc == nullptr)
+        return launch_cfg_impl<BLOCK_N, CTAS, EW, ABSMAX, kOutInt8>(a, s);
     if (a.Yq != nullptr || a.dbg_acc != nullptr) return launch_cfg_impl<BLOCK_N, CTAS, EW, ABSMAX, kOutFull>(a, s);
     if constexpr (CTAS == 2) {
         if (wants_direct_store<CTAS, EW>(a)) return launch_cfg_impl<BLOCK_N, CTAS, EW, ABSMAX, kOutDirect>(a, s);
