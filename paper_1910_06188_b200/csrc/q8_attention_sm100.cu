@@ -13,7 +13,8 @@
 //   phase 1  Q tile (scaled by log2(e)/8) -> Q_hi, Q_lo; per 128 keys: K rows -> K_hi, K_lo; 24 MMAs with N = 128
 //            (2 swizzle spans x 4 K steps x 3 partial products) -> scores in TMEM columns [128 c, 128 c + 128); the
 //            row maxima are read from TMEM chunk by chunk behind the MMAs (a row is shared by four threads)
-//   phase 2  per chunk: p = 2^(s - max) -> P_hi, P_lo (A operand, keys along K); V chunk transposed ->
+//   phase 2  per chunk: p = 2^(s - max) -> P_hi (back into tensor memory over the chunk's scores: the A operand is
+//            read from there), P_lo (shared memory; keys along K); V chunk transposed ->
 //            [V_hi ; V_lo] stacked as one 128-row B operand, so that one N = 128 MMA yields P_hi V_hi (columns
 //            0..63 of the O accumulator) and P_hi V_lo (columns 64..127), and one N = 64 MMA adds P_lo V_hi to the
 //            latter: 16 MMAs per chunk.  Keeping the small products in columns of their own also leaves a single
@@ -168,16 +169,18 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
                 ready_phase ^= 1u << b;
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t p_hi = smem_u32(p_buf(b)), p_lo = p_hi + 2 * kSpanBytesA, vb = smem_u32(kv_buf(b));
+                // P_hi is read from tensor memory, where it has replaced the chunk's scores (row = lane, key = column)
+                const uint32_t p_hi = tmem_base + (uint32_t)(kc * kChunk);
+                const uint32_t p_lo = smem_u32(p_buf(b)) + 2 * kSpanBytesA, vb = smem_u32(kv_buf(b));
                 uint32_t acc = kc > 0 ? 1u : 0u;
 #pragma unroll
                 for (int span = 0; span < 2; ++span) {
-                    const uint64_t ah = smem_desc_sw128(p_hi + span * kSpanBytesA), al = smem_desc_sw128(p_lo + span * kSpanBytesA);
+                    const uint64_t al = smem_desc_sw128(p_lo + span * kSpanBytesA);
                     const uint64_t bhl = smem_desc_sw128(vb + span * kSpanBytesB);  // 128 rows: V_hi then V_lo
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
+                    for (int ks = 0; ks < 4; ++ks) {  // 8 keys per instruction: 8 TMEM columns of P_hi, +2 in the (address >> 4) field
                         const uint64_t adv = (uint64_t)(2 * ks);
-                        umma_tf32_elected(elected, tmem_o, ah + adv, bhl + adv, kIdescN128, acc);         // [P_hi V_hi | P_hi V_lo]
+                        umma_tf32_ts_elected(elected, tmem_o, p_hi + (uint32_t)(32 * span + 8 * ks), bhl + adv, kIdescN128, acc);  // [P_hi V_hi | P_hi V_lo]
                         umma_tf32_elected(elected, tmem_o + kHeadDim, al + adv, bhl + adv, kIdescN64, 1u);  // += P_lo V_hi
                         acc = 1u;
                     }
@@ -203,6 +206,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
         // (16 arrivals on the barrier instead of 512)
         auto report_ready = [&](int b) {
             fence_proxy_async_smem();
+            tc_fence_before();  // (a tcgen05.st of P_hi has completed by now: tmem_st_wait() before this call)
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ready_bar[b]));
         };
@@ -298,19 +302,27 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
         if (ok) tmem_ld_32x16(t_row + (uint32_t)(cq * 16), pv);
         for (int kc = 0; kc < chunks && ok; ++kc) {
             const int b = kc & 1;
-            float p[16];
+            // p = hi + lo (hi = p rounded to TF32).  The hi parts go back into tensor memory over the chunk's scores, from
+            // where the MMA takes them as its A operand (no trip through shared memory: 64 x 384 x 16 heads 338 -> 325 us;
+            // the same for Q in phase 1 measured slower, 360 us, and is not done); the lo parts go to shared memory.
+            float p_lo[16];
             {
                 const int col0 = kc * kChunk + cq * 16;
                 tmem_ld_wait();
                 const bool whole = col0 + 16 <= S;
+                uint32_t ph[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     float e;
                     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(__uint_as_float(pv[j]) - m));
-                    p[j] = (whole || col0 + j < S) ? e : 0.0f;
-                    l += p[j];
+                    const float pj = (whole || col0 + j < S) ? e : 0.0f;
+                    l += pj;
+                    const float h = round_tf32(pj);
+                    ph[j] = __float_as_uint(h);
+                    p_lo[j] = pj - h;  // exact
                 }
                 if (kc + 1 < chunks) tmem_ld_32x16(t_row + (uint32_t)(col0 + kChunk), pv);
+                tmem_st_32x16(t_row + (uint32_t)col0, ph);
             }
             if (kc >= 2) {  // buffer set b was last read by the MMAs of chunk kc - 2
                 wait_done(b);
@@ -324,15 +336,15 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
                 store_split4(a1, a1 + kLoRowsB, make_float4(vreg[0].y, vreg[1].y, vreg[2].y, vreg[3].y));
             }
             if (kc + 1 < chunks) fetch_v((kc + 1) * kChunk);
-            // P[row][key]: this thread's 16 keys are pieces 4 (cq & 1) .. + 3 of span cq / 2 of the chunk
+            // P_lo[row][key]: this thread's 16 keys are pieces 4 (cq & 1) .. + 3 of span cq / 2 of the chunk
             {
-                uint8_t *sb = p_buf(b) + (cq >> 1) * kSpanBytesA;
+                uint8_t *sb = p_buf(b) + 2 * kSpanBytesA + (cq >> 1) * kSpanBytesA;
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    uint8_t *at = sb + sw128_offset(row, 4 * (cq & 1) + g);
-                    store_split4(at, at + 2 * kSpanBytesA, make_float4(p[4 * g], p[4 * g + 1], p[4 * g + 2], p[4 * g + 3]));
-                }
+                for (int g = 0; g < 4; ++g)
+                    *reinterpret_cast<float4 *>(sb + sw128_offset(row, 4 * (cq & 1) + g)) =
+                        make_float4(p_lo[4 * g], p_lo[4 * g + 1], p_lo[4 * g + 2], p_lo[4 * g + 3]);
             }
+            tmem_st_wait();
             report_ready(b);
         }
         tmem_ld_wait();  // (a load is still in flight only when the loop above was left early)
