@@ -8,8 +8,8 @@
 //
 // One CTA = 128 queries of one (sequence, head): 16 worker warps plus one warp that only issues MMAs.
 // All operands are staged by the workers themselves (global -> registers -> split -> shared memory in the
-// K-major 128-byte-swizzled layout the MMA reads); no TMA, no multicast.  Chunks of 64 keys go through two
-// buffer sets, so the MMAs of chunk c run while the workers prepare chunk c + 1:
+// K-major 128-byte-swizzled layout the MMA reads); no TMA, no multicast.  Chunks of keys go through two (phase 1)
+// or three (phase 2) buffer sets, so the MMAs of chunk c run while the workers prepare the chunks after it:
 //   phase 1  Q tile (scaled by log2(e)/8) -> Q_hi, Q_lo; per 128 keys: K rows -> K_hi, K_lo; 24 MMAs with N = 128
 //            (2 swizzle spans x 4 K steps x 3 partial products) -> scores in TMEM columns [128 c, 128 c + 128); the
 //            row maxima are read from TMEM chunk by chunk behind the MMAs (a row is shared by four threads)
@@ -43,14 +43,19 @@ constexpr int kSpanBytesB = 2 * kChunk * 128;  // ... of the 64-row operand, hi 
 constexpr int kLoRowsB = kChunk * 128;         // offset of the lo rows inside a B span
 constexpr int kBufQP = 4 * kSpanBytesA;        // {hi, lo} x 2 spans: Q, then P
 constexpr int kBufKV = 2 * kSpanBytesB;        // 2 spans x [hi ; lo]: K, then V^T
-constexpr int kAttnTcSmemBytes = 1024 + 2 * kBufQP + 2 * kBufKV;  // two buffer sets: 193 KB
+constexpr int kAttnTcSmemBytes = 1024 + 2 * kBufQP + 2 * kBufKV;  // 193 KB
+// Phase 2 needs V^T (hi and lo: kBufKV) and P_lo (half of kBufQP) per chunk: three such sets fill the same 192 KB
+// (against two sets: 325.7 -> 322.5 us for 64 x 384 x 16 heads).
+constexpr int kSets2 = 3;
+constexpr int kSet2Bytes = kBufKV + kBufQP / 2;
+static_assert(kSets2 * kSet2Bytes == 2 * kBufQP + 2 * kBufKV, "three phase-2 buffer sets use the whole allocation");
 // Phase 1 takes keys 128 at a time (N = 128 score MMAs: half as many instructions, each reading Q once for twice
-// the columns).  Its two K buffers of 64 KB ([hi 128 rows | lo 128 rows] per span) lie over the four phase-2
-// buffers behind Q.
+// the columns).  Its two K buffers of 64 KB ([hi 128 rows | lo 128 rows] per span) lie behind Q; phase 2 reuses the
+// whole allocation for its three buffer sets.
 constexpr int kBigChunk = 2 * kChunk;
 constexpr int kSpanBytesK = 2 * kBigChunk * 128;  // one span of a 128-key K buffer, hi rows then lo rows: 32 KB
 constexpr int kLoRowsK = kBigChunk * 128;
-static_assert(2 * (2 * kSpanBytesK) == 2 * kBufKV + kBufQP, "the two K buffers of phase 1 cover K/V 0, K/V 1 and P 1");
+static_assert(kBufQP + 2 * (2 * kSpanBytesK) == 2 * kBufQP + 2 * kBufKV, "Q and the two K buffers of phase 1 fill the allocation");
 
 // tcgen05.mma kind::tf32 instruction descriptor: D = F32, A = B = TF32, both K-major, M = 128.
 constexpr uint32_t kIdescBase = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kQTile >> 4) << 24);
@@ -96,11 +101,11 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     // [ Q, then P buffer 0 | K / V buffer 0 | K / V buffer 1 | P buffer 1 ]
     uint8_t *const q_buf = smem;
-    auto kv_buf = [&](int b) { return smem + kBufQP + b * kBufKV; };
-    auto k_buf = [&](int b) { return smem + kBufQP + b * (2 * kSpanBytesK); };  // phase 1 only
-    auto p_buf = [&](int b) { return smem + b * (kBufQP + 2 * kBufKV); };
-    __shared__ __align__(8) uint64_t ready_bar[2];  // workers -> MMA warp: the operands of a chunk are in place
-    __shared__ __align__(8) uint64_t done_bar[2];   // MMA warp -> workers: the MMAs of a chunk have completed
+    auto k_buf = [&](int b) { return smem + kBufQP + b * (2 * kSpanBytesK); };  // phase 1: two buffers behind Q
+    auto v_buf = [&](int b) { return smem + b * kSet2Bytes; };                  // phase 2: three sets of [V^T | P_lo]
+    auto plo_buf = [&](int b) { return smem + b * kSet2Bytes + kBufKV; };
+    __shared__ __align__(8) uint64_t ready_bar[kSets2];  // workers -> MMA warp: the operands of a chunk are in place
+    __shared__ __align__(8) uint64_t done_bar[kSets2];   // MMA warp -> workers: the MMAs of a chunk have completed
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float row_part[4][kQTile];  // per-row partial maxima, then partial sums, of the four column quarters
@@ -115,7 +120,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
     const int big_chunks = (S + kBigChunk - 1) / kBigChunk;
 
     if (tid == 0) {
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kSets2; ++b) {
             mbar_init(smem_u32(&ready_bar[b]), kWorkers / 32);  // one arrival per worker warp
             mbar_init(smem_u32(&done_bar[b]), 1);
         }
@@ -163,15 +168,14 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
                 }
                 umma_commit_elected(elected, smem_u32(&done_bar[b]));
             }
-            for (int kc = 0; kc < chunks && ok; ++kc) {  // O += P V of chunk kc
-                const int b = kc & 1;
+            for (int kc = 0, b = 0; kc < chunks && ok; ++kc, b = (b + 1 == kSets2 ? 0 : b + 1)) {  // O += P V of chunk kc
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&ready_bar[b]), (ready_phase >> b) & 1u, &abort_flag, status));
                 ready_phase ^= 1u << b;
                 if (!ok) break;
                 tc_fence_after();
                 // P_hi is read from tensor memory, where it has replaced the chunk's scores (row = lane, key = column)
                 const uint32_t p_hi = tmem_base + (uint32_t)(kc * kChunk);
-                const uint32_t p_lo = smem_u32(p_buf(b)) + 2 * kSpanBytesA, vb = smem_u32(kv_buf(b));
+                const uint32_t p_lo = smem_u32(plo_buf(b)), vb = smem_u32(v_buf(b));
                 uint32_t acc = kc > 0 ? 1u : 0u;
 #pragma unroll
                 for (int span = 0; span < 2; ++span) {
@@ -300,8 +304,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
         // exponentials are taken before the wait for the buffer set they will be stored into.
         uint32_t pv[16];
         if (ok) tmem_ld_32x16(t_row + (uint32_t)(cq * 16), pv);
-        for (int kc = 0; kc < chunks && ok; ++kc) {
-            const int b = kc & 1;
+        for (int kc = 0, b = 0; kc < chunks && ok; ++kc, b = (b + 1 == kSets2 ? 0 : b + 1)) {
             // p = hi + lo (hi = p rounded to TF32).  The hi parts go back into tensor memory over the chunk's scores, from
             // where the MMA takes them as its A operand (no trip through shared memory: 64 x 384 x 16 heads 338 -> 325 us;
             // the same for Q in phase 1 measured slower, 360 us, and is not done); the lo parts go to shared memory.
@@ -324,13 +327,13 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
                 if (kc + 1 < chunks) tmem_ld_32x16(t_row + (uint32_t)(col0 + kChunk), pv);
                 tmem_st_32x16(t_row + (uint32_t)col0, ph);
             }
-            if (kc >= 2) {  // buffer set b was last read by the MMAs of chunk kc - 2
+            if (kc >= kSets2) {  // buffer set b was last read by the MMAs of chunk kc - 3
                 wait_done(b);
                 if (!ok) break;
             }
             // V^T[d][key]: rows = features (64, hi block then lo block), K = keys of this chunk (2 spans of 32)
             {
-                uint8_t *sb = kv_buf(b) + (vkb >> 3) * kSpanBytesB;  // keys 4 vkb .. 4 vkb + 3: span vkb / 8, piece vkb % 8
+                uint8_t *sb = v_buf(b) + (vkb >> 3) * kSpanBytesB;  // keys 4 vkb .. 4 vkb + 3: span vkb / 8, piece vkb % 8
                 uint8_t *a0 = sb + sw128_offset(2 * vfp + 0, vkb & 7), *a1 = sb + sw128_offset(2 * vfp + 1, vkb & 7);
                 store_split4(a0, a0 + kLoRowsB, make_float4(vreg[0].x, vreg[1].x, vreg[2].x, vreg[3].x));
                 store_split4(a1, a1 + kLoRowsB, make_float4(vreg[0].y, vreg[1].y, vreg[2].y, vreg[3].y));
@@ -338,7 +341,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
             if (kc + 1 < chunks) fetch_v((kc + 1) * kChunk);
             // P_lo[row][key]: this thread's 16 keys are pieces 4 (cq & 1) .. + 3 of span cq / 2 of the chunk
             {
-                uint8_t *sb = p_buf(b) + 2 * kSpanBytesA + (cq >> 1) * kSpanBytesA;
+                uint8_t *sb = plo_buf(b) + (cq >> 1) * kSpanBytesA;
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
                     *reinterpret_cast<float4 *>(sb + sw128_offset(row, 4 * (cq & 1) + g)) =
@@ -350,7 +353,7 @@ attention_tc_kernel(const float *__restrict__ qkv, int S, int64_t H, float scale
         tmem_ld_wait();  // (a load is still in flight only when the loop above was left early)
         row_part[cq][row] = l;  // the row sums are exchanged while the last MMAs run
         worker_barrier();
-        for (int c = (chunks > 2 ? chunks - 2 : 0); c < chunks && ok; ++c) wait_done(c & 1);  // the last two chunks
+        for (int c = (chunks > kSets2 ? chunks - kSets2 : 0); c < chunks && ok; ++c) wait_done(c % kSets2);  // the last three chunks
 
         // ---------------- phase 3: ctx = (O_main + O_corr) / row sum
         if (ok) {  // (warp-uniform: the TMEM loads below are warp-wide instructions, only the stores depend on the row)
