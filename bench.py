@@ -696,8 +696,8 @@ def run_ours(args):
             "note": "an SM writes to L2 at no more than 32 bytes per clock (ncu: l1tex__m_l1tex2xbar_write_bytes peak), "
                     "whether by TMA store or by st.global, so the fp32 output of a layer occupies that port for "
                     "y_store_us_at_write_port (at the SM clock sampled in this run); measured kernel times are close to "
-                    "main_loop_only_us (the same kernel with the epilogue reduced to handing the accumulator back, a work "
-                    "copy, graph-replayed) plus that port time, i.e. the two do not overlap.  The main loop alone runs at "
+                    "main_loop_only_us (the same kernel with the epilogue reduced to handing the accumulator back, an "
+                    "experimental build, graph-replayed) plus that port time, i.e. the two do not overlap.  The main loop alone runs at "
                     "about three quarters of the issue-bound Int8 rate: TMA writes 64 B/clk/SM into shared memory while "
                     "the tensor cores read 64 B/clk/SM from it (with no loads the same loop takes 54.5 us on FFN2, with "
                     "only the B tiles 56.3, with both operands 66.4)",
